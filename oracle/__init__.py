@@ -1,0 +1,161 @@
+"""ctypes front end of the CPU oracle (``tsid_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product package imports this module;
+it is used by the tests, by the smoke check and by the bench's CPU-baseline leg.
+The arithmetic lives in the C file; this module only builds it with gcc,
+marshals numpy arrays and returns numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tsid_oracle.c")
+_LIB = os.path.join(_HERE, "libtsid_oracle.so")
+
+CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD = 0, 1, 2
+NORM_NONE, NORM_COUNT = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no fast-math).  Returns the .so path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.orc_bf16_round.restype = C.c_float
+        _lib.orc_bf16_round.argtypes = [C.c_float]
+        _lib.orc_clip_nested.restype = C.c_double
+        _lib.orc_clip_nested.argtypes = [C.c_double, C.c_double]
+    return _lib
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(C.POINTER(ct))
+
+
+def _coo(rows, cols, vals):
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    cols = np.ascontiguousarray(cols, dtype=np.int32)
+    vals = np.ascontiguousarray(vals, dtype=np.float32)
+    assert rows.shape == cols.shape == vals.shape and rows.ndim == 1
+    return rows, cols, vals
+
+
+def _fac(X, nrow, k):
+    X = np.ascontiguousarray(X, dtype=np.float32)
+    assert X.shape == (nrow, k), (X.shape, nrow, k)
+    return X
+
+
+def bf16_round(x: float) -> float:
+    return float(_L().orc_bf16_round(C.c_float(x)))
+
+
+def clip_nested(g: float, xi: float) -> float:
+    return float(_L().orc_clip_nested(g, xi))
+
+
+def residuals(m, n, k, rows, cols, vals, P, Q, bf16_emulate=False):
+    rows, cols, vals = _coo(rows, cols, vals)
+    P, Q = _fac(P, m, k), _fac(Q, n, k)
+    e = np.empty(rows.shape[0], dtype=np.float64)
+    _L().orc_residuals(C.c_int32(m), C.c_int32(n), C.c_int32(k), C.c_int64(rows.shape[0]),
+                       _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                       _p(P, C.c_float), _p(Q, C.c_float), C.c_int(int(bf16_emulate)),
+                       _p(e, C.c_double))
+    return e
+
+
+@dataclass
+class Step:
+    GP: np.ndarray  # raw sums E Q, float64 (m, k)
+    GQ: np.ndarray  # raw sums E^T P, float64 (n, k)
+    DP: np.ndarray  # clipped direction, float64
+    DQ: np.ndarray
+    P: np.ndarray   # updated factors, float32
+    Q: np.ndarray
+
+
+def grad_step(m, n, k, rows, cols, vals, P, Q, eta, lam, xi,
+              clip=CLIP_NONE, norm_p=NORM_NONE, norm_q=NORM_NONE, bf16_emulate=False) -> Step:
+    rows, cols, vals = _coo(rows, cols, vals)
+    P, Q = _fac(P, m, k), _fac(Q, n, k)
+    GP = np.empty((m, k)); GQ = np.empty((n, k)); DP = np.empty((m, k)); DQ = np.empty((n, k))
+    Pn = np.empty((m, k), dtype=np.float32); Qn = np.empty((n, k), dtype=np.float32)
+    _L().orc_grad_step(C.c_int32(m), C.c_int32(n), C.c_int32(k), C.c_int64(rows.shape[0]),
+                       _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                       _p(P, C.c_float), _p(Q, C.c_float),
+                       C.c_double(eta), C.c_double(lam), C.c_double(xi),
+                       C.c_int(clip), C.c_int(norm_p), C.c_int(norm_q), C.c_int(int(bf16_emulate)),
+                       _p(GP, C.c_double), _p(GQ, C.c_double), _p(DP, C.c_double), _p(DQ, C.c_double),
+                       _p(Pn, C.c_float), _p(Qn, C.c_float))
+    return Step(GP, GQ, DP, DQ, Pn, Qn)
+
+
+def loss(m, n, k, rows, cols, vals, P, Q, lam, bf16_emulate=False):
+    """Returns (SSE, objective)."""
+    rows, cols, vals = _coo(rows, cols, vals)
+    P, Q = _fac(P, m, k), _fac(Q, n, k)
+    sse = C.c_double(0.0); obj = C.c_double(0.0)
+    _L().orc_loss(C.c_int32(m), C.c_int32(n), C.c_int32(k), C.c_int64(rows.shape[0]),
+                  _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                  _p(P, C.c_float), _p(Q, C.c_float), C.c_double(lam), C.c_int(int(bf16_emulate)),
+                  C.byref(sse), C.byref(obj))
+    return sse.value, obj.value
+
+
+def fit(m, n, k, rows, cols, vals, P, Q, epochs, eta, lam, xi,
+        clip=CLIP_NONE, norm_p=NORM_NONE, norm_q=NORM_NONE, bf16_emulate=False, history=True):
+    """Runs `epochs` steps on copies of P, Q.  Returns (P, Q, sse_history or None)."""
+    rows, cols, vals = _coo(rows, cols, vals)
+    P = _fac(P, m, k).copy(); Q = _fac(Q, n, k).copy()
+    hist = np.empty(epochs + 1, dtype=np.float64) if history else None
+    _L().orc_fit(C.c_int32(m), C.c_int32(n), C.c_int32(k), C.c_int64(rows.shape[0]),
+                 _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                 _p(P, C.c_float), _p(Q, C.c_float), C.c_int32(epochs),
+                 C.c_double(eta), C.c_double(lam), C.c_double(xi),
+                 C.c_int(clip), C.c_int(norm_p), C.c_int(norm_q), C.c_int(int(bf16_emulate)),
+                 _p(hist, C.c_double) if history else None)
+    return P, Q, hist
+
+
+@dataclass
+class Layout:
+    row_ptr: np.ndarray  # int64 (m+1)
+    col_idx: np.ndarray  # int32 (nnz), CSR order
+    val_csr: np.ndarray  # float32
+    col_ptr: np.ndarray  # int64 (n+1)
+    row_idx: np.ndarray  # int32 (nnz), CSC order
+    val_csc: np.ndarray  # float32
+    perm: np.ndarray     # uint32: CSR position of CSC entry t
+
+
+def layout(m, n, rows, cols, vals) -> Layout:
+    rows, cols, vals = _coo(rows, cols, vals)
+    nnz = rows.shape[0]
+    out = Layout(np.empty(m + 1, np.int64), np.empty(nnz, np.int32), np.empty(nnz, np.float32),
+                 np.empty(n + 1, np.int64), np.empty(nnz, np.int32), np.empty(nnz, np.float32),
+                 np.empty(nnz, np.uint32))
+    _L().orc_layout(C.c_int32(m), C.c_int32(n), C.c_int64(nnz),
+                    _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                    _p(out.row_ptr, C.c_int64), _p(out.col_idx, C.c_int32), _p(out.val_csr, C.c_float),
+                    _p(out.col_ptr, C.c_int64), _p(out.row_idx, C.c_int32), _p(out.val_csc, C.c_float),
+                    _p(out.perm, C.c_uint32))
+    return out

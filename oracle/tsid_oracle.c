@@ -1,0 +1,256 @@
+/*
+ * TSID template-recovery oracle: TEST INFRASTRUCTURE, not product code.
+ *
+ * A plain, slow, single-threaded CPU statement of what one full-batch gradient
+ * step of the masked low-rank (regularised matrix factorisation, RMF) objective
+ * computes.  All sums are taken in double precision, looping over the COO
+ * triples in input order.  No blocking, no fusion, no reordering.  It shares no
+ * code with the CUDA library; only tests, the smoke check and the bench's CPU
+ * baseline leg may call it.
+ *
+ * Passages followed (paper sections / equations):
+ *   - objective: Sec. 3.2, Eq. (rmf-obj):
+ *       L(P,Q) = sum_{(i,j) in Omega} (r_ij - p_i . q_j)^2 + lambda (|P|_F^2 + |Q|_F^2)
+ *   - per-entry gradients: Sec. 5.1, Eqs. (update-p), (update-q):
+ *       grad_p = -2 e q + 2 lambda p,   grad_q = -2 e p + 2 lambda q,  e = r - p.q
+ *   - aggregated update and the 1/n normalisation: Sec. 5.1, Eq. 9
+ *   - asymmetric clipping min(max(xi, -g), g): Sec. 5.3 (unnumbered equation)
+ *
+ * Readings taken where the paper is ambiguous (all listed in the design notes):
+ *   - the symbol added to the factors in Eq. 9 is the step DIRECTION
+ *       D = -grad L = 2 G / s - 2 lambda x,   G_P = E Q,  G_Q = E^T P,
+ *     E the sparse residual matrix; the update is x + eta * D;
+ *   - the "n" in the 1/n factor is the number of observed entries that
+ *     contribute to that factor row (norm = COUNT), s = max(1, count);
+ *     norm = NONE gives s = 1 which is exactly -grad of Eq. (rmf-obj);
+ *   - the regulariser enters once per factor row (-2 lambda x), not once per entry;
+ *   - the clip acts on the aggregated, normalised, regularised direction;
+ *     CLIP_ASYM_STEP: D <- min(max(xi,-D), D)   (caps increases at eta*xi);
+ *     CLIP_ASYM_GRAD: the same formula applied to the loss gradient g = -D,
+ *     then the step is -eta * clip(g);
+ *   - both factor updates use the same residuals (Jacobi, simultaneous).
+ *
+ * Pins: every function below is pinned by tests marked "not gpu" (hand-worked
+ * 3x2 and 8x6 examples stored as golden text, finite differences of the loss,
+ * zero gradient at the true factors, the dense special case against numpy,
+ * the trace identity, the single-entry case, monotone loss, closed form of the
+ * clip, and the layout against numpy.lexsort).  The bf16 path has no exact pin
+ * beyond the emulation switch (inputs rounded to bf16, round-to-nearest-even):
+ * the rounding function itself is pinned against a table of hand-derived bit
+ * patterns.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORC_CLIP_NONE = 0, ORC_CLIP_ASYM_STEP = 1, ORC_CLIP_ASYM_GRAD = 2 };
+enum { ORC_NORM_NONE = 0, ORC_NORM_COUNT = 1 };
+
+/* Round a float to the nearest bfloat16 (ties to even) and return it as float.
+ * bfloat16 keeps the top 16 bits of the IEEE-754 binary32 pattern. */
+float orc_bf16_round(float x) {
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  if ((u & 0x7f800000u) == 0x7f800000u) { /* inf / nan: truncate, keep nan a nan */
+    if (u & 0x007fffffu) u |= 0x00400000u;
+    u &= 0xffff0000u;
+  } else {
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    u &= 0xffff0000u;
+  }
+  float y;
+  memcpy(&y, &u, 4);
+  return y;
+}
+
+/* Sec. 5.3: the nested clip, written exactly as printed. */
+double orc_clip_nested(double g, double xi) {
+  double a = (xi > -g) ? xi : -g;   /* max(xi, -g) */
+  return (a < g) ? a : g;           /* min(.., g)  */
+}
+
+static double read_factor(const float *X, int64_t idx, int bf16_emulate) {
+  float v = X[idx];
+  if (bf16_emulate) v = orc_bf16_round(v);
+  return (double)v;
+}
+
+/* e_t = r_t - sum_l P[i_t,l] Q[j_t,l], t in input order (Eqs. update-p/q: the
+ * factor (R_ji - p_j q_i^T)). */
+void orc_residuals(int32_t m, int32_t n, int32_t k, int64_t nnz,
+                   const int32_t *rows, const int32_t *cols, const float *vals,
+                   const float *P, const float *Q, int bf16_emulate, double *e_out) {
+  (void)m; (void)n;
+  for (int64_t t = 0; t < nnz; ++t) {
+    int64_t i = rows[t], j = cols[t];
+    double dot = 0.0;
+    for (int32_t l = 0; l < k; ++l)
+      dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
+    e_out[t] = (double)vals[t] - dot;
+  }
+}
+
+/* Raw gradient sums G_P = E Q (m x k), G_Q = E^T P (n x k) and the per-row /
+ * per-column observation counts.  Outputs are overwritten. */
+void orc_grad_sums(int32_t m, int32_t n, int32_t k, int64_t nnz,
+                   const int32_t *rows, const int32_t *cols, const float *vals,
+                   const float *P, const float *Q, int bf16_emulate,
+                   double *GP, double *GQ, int64_t *cntP, int64_t *cntQ) {
+  memset(GP, 0, sizeof(double) * (size_t)m * k);
+  memset(GQ, 0, sizeof(double) * (size_t)n * k);
+  memset(cntP, 0, sizeof(int64_t) * (size_t)m);
+  memset(cntQ, 0, sizeof(int64_t) * (size_t)n);
+  for (int64_t t = 0; t < nnz; ++t) {
+    int64_t i = rows[t], j = cols[t];
+    double dot = 0.0;
+    for (int32_t l = 0; l < k; ++l)
+      dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
+    double e = (double)vals[t] - dot;
+    for (int32_t l = 0; l < k; ++l) {
+      GP[i * k + l] += e * read_factor(Q, j * k + l, bf16_emulate);
+      GQ[j * k + l] += e * read_factor(P, i * k + l, bf16_emulate);
+    }
+    cntP[i] += 1;
+    cntQ[j] += 1;
+  }
+}
+
+/* Direction for one factor matrix: D = 2 G / s - 2 lambda X, then the clip.
+ * X is the fp32 master value (never the bf16-rounded one). */
+static void direction(int64_t nrow, int32_t k, const double *G, const int64_t *cnt,
+                      const float *X, double lambda, double xi, int clip, int norm,
+                      double *D) {
+  for (int64_t r = 0; r < nrow; ++r) {
+    double s = 1.0;
+    if (norm == ORC_NORM_COUNT) s = (cnt[r] > 1) ? (double)cnt[r] : 1.0;
+    for (int32_t l = 0; l < k; ++l) {
+      double d = 2.0 * G[r * k + l] / s - 2.0 * lambda * (double)X[r * k + l];
+      if (clip == ORC_CLIP_ASYM_STEP) {
+        d = orc_clip_nested(d, xi);
+      } else if (clip == ORC_CLIP_ASYM_GRAD) {
+        d = -orc_clip_nested(-d, xi);
+      }
+      D[r * k + l] = d;
+    }
+  }
+}
+
+/* One full-batch step.  P, Q are read; P_new, Q_new (fp32, may alias nothing)
+ * receive x + eta D rounded once to fp32.  GP, GQ (double, m*k / n*k) receive
+ * the raw sums; DP, DQ (double) the clipped directions.  Any of GP/GQ/DP/DQ
+ * must be valid buffers (the caller allocates). */
+void orc_grad_step(int32_t m, int32_t n, int32_t k, int64_t nnz,
+                   const int32_t *rows, const int32_t *cols, const float *vals,
+                   const float *P, const float *Q,
+                   double eta, double lambda, double xi,
+                   int clip, int norm_p, int norm_q, int bf16_emulate,
+                   double *GP, double *GQ, double *DP, double *DQ,
+                   float *P_new, float *Q_new) {
+  int64_t *cntP = (int64_t *)malloc(sizeof(int64_t) * (size_t)(m > 0 ? m : 1));
+  int64_t *cntQ = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n > 0 ? n : 1));
+  orc_grad_sums(m, n, k, nnz, rows, cols, vals, P, Q, bf16_emulate, GP, GQ, cntP, cntQ);
+  direction(m, k, GP, cntP, P, lambda, xi, clip, norm_p, DP);
+  direction(n, k, GQ, cntQ, Q, lambda, xi, clip, norm_q, DQ);
+  for (int64_t a = 0; a < (int64_t)m * k; ++a) P_new[a] = (float)((double)P[a] + eta * DP[a]);
+  for (int64_t a = 0; a < (int64_t)n * k; ++a) Q_new[a] = (float)((double)Q[a] + eta * DQ[a]);
+  free(cntP);
+  free(cntQ);
+}
+
+/* SSE = sum e^2 and obj = SSE + lambda (|P|_F^2 + |Q|_F^2), Eq. (rmf-obj). */
+void orc_loss(int32_t m, int32_t n, int32_t k, int64_t nnz,
+              const int32_t *rows, const int32_t *cols, const float *vals,
+              const float *P, const float *Q, double lambda, int bf16_emulate,
+              double *sse_out, double *obj_out) {
+  double sse = 0.0;
+  for (int64_t t = 0; t < nnz; ++t) {
+    int64_t i = rows[t], j = cols[t];
+    double dot = 0.0;
+    for (int32_t l = 0; l < k; ++l)
+      dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
+    double e = (double)vals[t] - dot;
+    sse += e * e;
+  }
+  double reg = 0.0;
+  for (int64_t a = 0; a < (int64_t)m * k; ++a) reg += (double)P[a] * (double)P[a];
+  for (int64_t a = 0; a < (int64_t)n * k; ++a) reg += (double)Q[a] * (double)Q[a];
+  *sse_out = sse;
+  *obj_out = sse + lambda * reg;
+}
+
+/* `epochs` steps in place on P, Q.  If sse_hist is non-null it receives
+ * epochs+1 values: the SSE before the first step and after every step. */
+void orc_fit(int32_t m, int32_t n, int32_t k, int64_t nnz,
+             const int32_t *rows, const int32_t *cols, const float *vals,
+             float *P, float *Q, int32_t epochs,
+             double eta, double lambda, double xi,
+             int clip, int norm_p, int norm_q, int bf16_emulate, double *sse_hist) {
+  size_t mk = (size_t)m * k, nk = (size_t)n * k;
+  double *GP = (double *)malloc(sizeof(double) * (mk ? mk : 1));
+  double *GQ = (double *)malloc(sizeof(double) * (nk ? nk : 1));
+  double *DP = (double *)malloc(sizeof(double) * (mk ? mk : 1));
+  double *DQ = (double *)malloc(sizeof(double) * (nk ? nk : 1));
+  float *Pn = (float *)malloc(sizeof(float) * (mk ? mk : 1));
+  float *Qn = (float *)malloc(sizeof(float) * (nk ? nk : 1));
+  double obj;
+  if (sse_hist) orc_loss(m, n, k, nnz, rows, cols, vals, P, Q, lambda, bf16_emulate, &sse_hist[0], &obj);
+  for (int32_t ep = 0; ep < epochs; ++ep) {
+    orc_grad_step(m, n, k, nnz, rows, cols, vals, P, Q, eta, lambda, xi, clip, norm_p, norm_q,
+                  bf16_emulate, GP, GQ, DP, DQ, Pn, Qn);
+    memcpy(P, Pn, sizeof(float) * mk);
+    memcpy(Q, Qn, sizeof(float) * nk);
+    if (sse_hist)
+      orc_loss(m, n, k, nnz, rows, cols, vals, P, Q, lambda, bf16_emulate, &sse_hist[ep + 1], &obj);
+  }
+  free(GP); free(GQ); free(DP); free(DQ); free(Pn); free(Qn);
+}
+
+/* Layout: order entry ids by (row, col, input position) -> CSR and by
+ * (col, row, input position) -> CSC; perm[t] = CSR position of CSC entry t.
+ * The order is unique when Omega is a set; ties (duplicates) break by input
+ * position. */
+typedef struct { int32_t a, b; int64_t id; } orc_key_t;
+
+static int key_cmp(const void *x, const void *y) {
+  const orc_key_t *u = (const orc_key_t *)x, *v = (const orc_key_t *)y;
+  if (u->a != v->a) return (u->a < v->a) ? -1 : 1;
+  if (u->b != v->b) return (u->b < v->b) ? -1 : 1;
+  if (u->id != v->id) return (u->id < v->id) ? -1 : 1;
+  return 0;
+}
+
+void orc_layout(int32_t m, int32_t n, int64_t nnz,
+                const int32_t *rows, const int32_t *cols, const float *vals,
+                int64_t *row_ptr, int32_t *col_idx, float *val_csr,
+                int64_t *col_ptr, int32_t *row_idx, float *val_csc, uint32_t *perm) {
+  orc_key_t *keys = (orc_key_t *)malloc(sizeof(orc_key_t) * (size_t)(nnz > 0 ? nnz : 1));
+  int64_t *csr_pos = (int64_t *)malloc(sizeof(int64_t) * (size_t)(nnz > 0 ? nnz : 1));
+  /* CSR */
+  for (int64_t t = 0; t < nnz; ++t) { keys[t].a = rows[t]; keys[t].b = cols[t]; keys[t].id = t; }
+  qsort(keys, (size_t)nnz, sizeof(orc_key_t), key_cmp);
+  for (int64_t i = 0; i <= m; ++i) row_ptr[i] = 0;
+  for (int64_t p = 0; p < nnz; ++p) {
+    int64_t t = keys[p].id;
+    col_idx[p] = cols[t];
+    val_csr[p] = vals[t];
+    csr_pos[t] = p;
+    row_ptr[(int64_t)rows[t] + 1] += 1;
+  }
+  for (int64_t i = 0; i < m; ++i) row_ptr[i + 1] += row_ptr[i];
+  /* CSC */
+  for (int64_t t = 0; t < nnz; ++t) { keys[t].a = cols[t]; keys[t].b = rows[t]; keys[t].id = t; }
+  qsort(keys, (size_t)nnz, sizeof(orc_key_t), key_cmp);
+  for (int64_t j = 0; j <= n; ++j) col_ptr[j] = 0;
+  for (int64_t p = 0; p < nnz; ++p) {
+    int64_t t = keys[p].id;
+    row_idx[p] = rows[t];
+    val_csc[p] = vals[t];
+    perm[p] = (uint32_t)csr_pos[t];
+    col_ptr[(int64_t)cols[t] + 1] += 1;
+  }
+  for (int64_t j = 0; j < n; ++j) col_ptr[j + 1] += col_ptr[j];
+  free(keys);
+  free(csr_pos);
+}
