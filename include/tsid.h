@@ -1,0 +1,171 @@
+/*
+ * tsid.h - C ABI of the B200 (sm_100a) template-recovery factorization.
+ *
+ * Problem (Sec. 1 and Def. 1 of the paper; Sec. 3.2, Eq. (rmf-obj)): a template
+ * R in R^{m x n} is known on an index set Omega (|Omega| = nnz).  Stage I of
+ * TSID matrix completion fits factors P in R^{m x k}, Q in R^{n x k} to
+ *
+ *     L(P, Q) = sum_{(i,j) in Omega} (r_ij - p_i . q_j)^2 + lambda (|P|_F^2 + |Q|_F^2)
+ *
+ * by full-batch gradient steps.  One step (Sec. 5.1, Eqs. (update-p), (update-q), Eq. 9;
+ * Sec. 5.3 for the clip) computes, from the SAME (P, Q) for both sides:
+ *
+ *     e_ij = r_ij - p_i . q_j                          for (i,j) in Omega
+ *     G_P  = E Q   (m x k),   G_Q = E^T P   (n x k)    E = sparse residual matrix
+ *     D_P[i,:] = 2 G_P[i,:] / s_i  - 2 lambda P[i,:]   s_i  = 1 or max(1, |Omega_i|)
+ *     D_Q[j,:] = 2 G_Q[j,:] / s'_j - 2 lambda Q[j,:]   s'_j = 1 or max(1, |Omega^j|)
+ *     D <- clip(D)                                     ASYM_STEP: min(D, xi)
+ *     P <- P + eta D_P,   Q <- Q + eta D_Q
+ *
+ * The sums are accumulated warp -> block -> grid in a fixed order (no floating
+ * point atomics): identical inputs give bitwise identical outputs.
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The library
+ *     never allocates device memory: all device state lives in the caller's
+ *     `workspace` (size from tsid_workspace_bytes), which must stay valid and
+ *     untouched until tsid_destroy.  The handle owns host bookkeeping only.
+ *   - P is row-major m x k fp32, Q is row-major n x k fp32, caller-owned, 16-byte
+ *     aligned, updated in place.
+ *   - All work is enqueued on cfg.stream.  tsid_grad_step and tsid_fit with
+ *     loss_every == 0 do not synchronise; tsid_template_create, tsid_loss,
+ *     tsid_fit with loss_every > 0 and tsid_check synchronise the stream.
+ *   - Every call returns a status; nothing throws, aborts or traps.  Argument
+ *     errors are detected before any launch.  tsid_last_error gives a message.
+ *   - Limits: 1 <= k <= 256, k a multiple of 4 (TSID_F32) or 8 (TSID_BF16_SHADOW);
+ *     0 <= nnz <= 2^31 - 1; m, n >= 1.
+ */
+#ifndef TSID_H_
+#define TSID_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tsid_template tsid_template_t; /* opaque */
+
+typedef enum {
+  TSID_OK = 0,
+  TSID_ERR_INVALID_ARG = 1,  /* null pointer, bad size, bad enum, misaligned pointer      */
+  TSID_ERR_INDEX_RANGE = 2,  /* a row index outside [0,m) or column index outside [0,n)   */
+  TSID_ERR_DUPLICATE = 3,    /* TSID_VALIDATE: the same (row, col) appears twice          */
+  TSID_ERR_UNSORTED = 4,     /* TSID_INPUT_ROW_SORTED promised but the input is not       */
+  TSID_ERR_OOM = 5,          /* workspace smaller than tsid_workspace_bytes               */
+  TSID_ERR_CUDA = 6,         /* a CUDA runtime call failed (message in tsid_last_error)   */
+  TSID_ERR_UNSUPPORTED = 7,  /* configuration outside the limits above                    */
+  TSID_ERR_NONFINITE = 8     /* an updated factor became inf/nan (reported by tsid_check, */
+                             /* tsid_loss and tsid_fit with loss_every > 0)               */
+} tsid_status_t;
+
+/* Storage precision of the factor values the two gradient passes READ.  The
+ * caller's P, Q are always the fp32 master copy.  TSID_BF16_SHADOW keeps a
+ * bfloat16 copy (round to nearest even) refreshed by the update kernel; products
+ * are exact in fp32 and all sums are fp32 (Sec. 5.1 mixed precision: 16-bit
+ * multiplicands, 32-bit accumulation). */
+typedef enum { TSID_F32 = 0, TSID_BF16_SHADOW = 1 } tsid_precision_t;
+
+/* TSID_PATH_SPARSE: CSR/CSC gather-reduce passes (HBM bound).
+ * TSID_PATH_DENSE_TC: tcgen05 masked-GEMM variant (Sec. 5.1, "Regularizing Sparse RMF
+ * Updates for Tensor Cores"): P Q^T, then E Q and E^T P with bf16 operands and fp32
+ * accumulation; requires TSID_BF16_SHADOW, k a multiple of 16 and m, n multiples of 128.
+ * TSID_PATH_AUTO picks DENSE_TC when the template qualifies and nnz / (m n) >= 0.05. */
+typedef enum { TSID_PATH_AUTO = 0, TSID_PATH_SPARSE = 1, TSID_PATH_DENSE_TC = 2 } tsid_path_t;
+
+/* Sec. 5.3.  ASYM_STEP (default reading): D <- min(max(xi, -D), D) = min(D, xi): increases
+ * of a coordinate are capped at eta*xi, decreases are free.  ASYM_GRAD: the same formula
+ * applied to the loss gradient g = -D, i.e. D <- max(D, -xi). */
+typedef enum { TSID_CLIP_NONE = 0, TSID_CLIP_ASYM_STEP = 1, TSID_CLIP_ASYM_GRAD = 2 } tsid_clip_t;
+
+/* Eq. 9's 1/n factor: divide the summed gradient of a factor row by the number of
+ * observed entries that contribute to it (COUNT) or not at all (NONE). */
+typedef enum { TSID_NORM_NONE = 0, TSID_NORM_COUNT = 1 } tsid_norm_t;
+
+enum {
+  TSID_VALIDATE = 1u,         /* also check Omega for duplicate (row, col) pairs            */
+  TSID_INPUT_ROW_SORTED = 2u  /* promise: COO is sorted by (row, col); checked, skips a sort */
+};
+
+typedef struct {
+  int32_t m, n, k;
+  int64_t nnz;
+  int32_t precision; /* tsid_precision_t */
+  int32_t path;      /* tsid_path_t      */
+  float eta, lambda, xi;
+  int32_t clip;      /* tsid_clip_t */
+  int32_t norm_p;    /* tsid_norm_t */
+  int32_t norm_q;    /* tsid_norm_t */
+  uint32_t flags;
+  void *stream;           /* cudaStream_t owned by the caller (0 = legacy default stream) */
+  void *workspace;        /* DEVICE memory owned by the caller, 256-byte aligned          */
+  size_t workspace_bytes; /* its size                                                     */
+} tsid_config_t;
+
+/* Bytes of device workspace a template with cfg's m, n, k, nnz, precision and path needs.
+ * Reads only those fields.  Host-only, no CUDA call. */
+tsid_status_t tsid_workspace_bytes(const tsid_config_t *cfg, size_t *h_bytes_out);
+
+/* Layout pass + handle creation.  d_rows, d_cols (int32[nnz]) and d_vals (fp32[nnz]) are
+ * the COO triples of Omega on the DEVICE, in any order; they are only read, and may be
+ * freed when the call returns (it synchronises cfg.stream).  Builds in the workspace:
+ * CSR sorted by (row, col), CSC sorted by (col, row), perm (CSC position -> CSR position),
+ * the equal-length work segments of both passes, gradient / shadow / partial buffers.
+ * Duplicates, when not rejected by TSID_VALIDATE, are each counted; ties keep input order.
+ * On error *out is NULL. */
+tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_rows,
+                                   const int32_t *d_cols, const float *d_vals,
+                                   tsid_template_t **out);
+
+/* One full-batch step, in place on d_P (m x k) and d_Q (n x k).  If d_gradP / d_gradQ are
+ * non-null they receive the raw sums G_P = E Q (m x k) and G_Q = E^T P (n x k), fp32,
+ * computed from the factors as they were BEFORE the update.  Asynchronous. */
+tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *d_gradP_or_null,
+                             float *d_gradQ_or_null);
+
+/* `epochs` steps in place.  loss_every > 0: after every loss_every-th step (and before the
+ * first) the SSE is computed and stored in h_sse_history_or_null (host, capacity
+ * 1 + epochs / loss_every doubles); this synchronises.  loss_every == 0: asynchronous. */
+tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epochs,
+                       int32_t loss_every, double *h_sse_history_or_null);
+
+/* SSE = sum_Omega e^2 and objective = SSE + lambda (|P|_F^2 + |Q|_F^2) (Eq. (rmf-obj)).
+ * Residuals are taken at the template's precision (bf16 shadows if so configured), squares
+ * are summed in double in a fixed order; the norms use the fp32 values.  Synchronises. */
+tsid_status_t tsid_loss(tsid_template_t *t, const float *d_P, const float *d_Q, double *h_sse,
+                        double *h_objective);
+
+/* Synchronises the stream and reports a pending device-side condition
+ * (TSID_ERR_NONFINITE, TSID_ERR_CUDA) or TSID_OK. */
+tsid_status_t tsid_check(tsid_template_t *t);
+
+/* Releases the host handle.  The workspace belongs to the caller.  NULL is accepted. */
+tsid_status_t tsid_destroy(tsid_template_t *t);
+
+/* ---- debug / test surface ------------------------------------------------------------ */
+
+/* Device pointers into the workspace (valid until destroy): row_ptr int64[m+1], col_idx
+ * int32[nnz] and val_csr fp32[nnz] in CSR order; col_ptr int64[n+1], row_idx int32[nnz] and
+ * val_csc fp32[nnz] in CSC order; perm uint32[nnz].  Any out pointer may be NULL. */
+tsid_status_t tsid_get_layout(tsid_template_t *t, const int64_t **d_row_ptr,
+                              const int32_t **d_col_idx, const float **d_val_csr,
+                              const int64_t **d_col_ptr, const int32_t **d_row_idx,
+                              const float **d_val_csc, const uint32_t **d_perm);
+
+/* e in CSR order (fp32[nnz], device), at the template's precision.  Asynchronous. */
+tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *d_Q,
+                             float *d_e_csr);
+
+/* Which path the handle runs (tsid_path_t, never AUTO) and how many kernels one
+ * tsid_grad_step launches. */
+tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
+
+/* Message of the last failing call on this handle (or of the last failing create when
+ * t == NULL).  Never NULL; valid until the next call on the same handle / thread. */
+const char *tsid_last_error(const tsid_template_t *t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSID_H_ */

@@ -1,0 +1,224 @@
+"""Thin ctypes layer over libtsid.so: argument marshalling only.
+
+Names and arguments follow include/tsid.h.  Device memory and streams come from
+PyTorch tensors (``.data_ptr()``); every step of the path runs in the library's
+kernels.  A missing library is an error: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtsid.so")
+
+TSID_OK = 0
+STATUS_NAMES = ["TSID_OK", "TSID_ERR_INVALID_ARG", "TSID_ERR_INDEX_RANGE", "TSID_ERR_DUPLICATE",
+                "TSID_ERR_UNSORTED", "TSID_ERR_OOM", "TSID_ERR_CUDA", "TSID_ERR_UNSUPPORTED",
+                "TSID_ERR_NONFINITE"]
+(TSID_ERR_INVALID_ARG, TSID_ERR_INDEX_RANGE, TSID_ERR_DUPLICATE, TSID_ERR_UNSORTED, TSID_ERR_OOM,
+ TSID_ERR_CUDA, TSID_ERR_UNSUPPORTED, TSID_ERR_NONFINITE) = range(1, 9)
+TSID_F32, TSID_BF16_SHADOW = 0, 1
+TSID_PATH_AUTO, TSID_PATH_SPARSE, TSID_PATH_DENSE_TC = 0, 1, 2
+TSID_CLIP_NONE, TSID_CLIP_ASYM_STEP, TSID_CLIP_ASYM_GRAD = 0, 1, 2
+TSID_NORM_NONE, TSID_NORM_COUNT = 0, 1
+TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
+
+# every symbol include/tsid.h declares
+EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",
+           "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
+           "tsid_last_error"]
+
+
+class TsidConfig(C.Structure):
+    _fields_ = [("m", C.c_int32), ("n", C.c_int32), ("k", C.c_int32), ("nnz", C.c_int64),
+                ("precision", C.c_int32), ("path", C.c_int32),
+                ("eta", C.c_float), ("lam", C.c_float), ("xi", C.c_float),
+                ("clip", C.c_int32), ("norm_p", C.c_int32), ("norm_q", C.c_int32),
+                ("flags", C.c_uint32), ("stream", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_size_t)]
+
+
+class TsidError(RuntimeError):
+    def __init__(self, status, message):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__("%s: %s" % (name, message))
+
+
+_lib = None
+
+
+def lib():
+    """Loads libtsid.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libtsid.so is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp = C.c_void_p
+        L.tsid_workspace_bytes.argtypes = [C.POINTER(TsidConfig), C.POINTER(C.c_size_t)]
+        L.tsid_template_create.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, C.POINTER(vp)]
+        L.tsid_grad_step.argtypes = [vp, vp, vp, vp, vp]
+        L.tsid_fit.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.tsid_loss.argtypes = [vp, vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.tsid_check.argtypes = [vp]
+        L.tsid_destroy.argtypes = [vp]
+        L.tsid_get_layout.argtypes = [vp] + [C.POINTER(vp)] * 7
+        L.tsid_residuals.argtypes = [vp, vp, vp, vp]
+        L.tsid_get_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.tsid_last_error.argtypes = [vp]
+        L.tsid_last_error.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "tsid_last_error":
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check_tensor(t, dtype, numel, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()
+            and t.numel() == numel):
+        raise ValueError("%s must be a contiguous CUDA tensor of %s with %d elements" % (name, dtype, numel))
+
+
+def make_config(m, n, k, nnz, precision=TSID_F32, path=TSID_PATH_AUTO, eta=0.01, lam=0.0, xi=0.1,
+                clip=TSID_CLIP_NONE, norm_p=TSID_NORM_NONE, norm_q=TSID_NORM_NONE, flags=0) -> TsidConfig:
+    return TsidConfig(m, n, k, nnz, precision, path, eta, lam, xi, clip, norm_p, norm_q, flags, None, None, 0)
+
+
+def tsid_workspace_bytes(cfg: TsidConfig) -> int:
+    out = C.c_size_t(0)
+    st = lib().tsid_workspace_bytes(C.byref(cfg), C.byref(out))
+    if st != TSID_OK:
+        raise TsidError(st, lib().tsid_last_error(None).decode())
+    return out.value
+
+
+class Template:
+    """Owns the workspace tensor and the handle of one template (tsid_template_create ... tsid_destroy)."""
+
+    def __init__(self, cfg: TsidConfig, rows: torch.Tensor, cols: torch.Tensor, vals: torch.Tensor,
+                 stream: torch.cuda.Stream | None = None):
+        L = lib()
+        nnz = int(cfg.nnz)
+        _check_tensor(rows, torch.int32, nnz, "rows")
+        _check_tensor(cols, torch.int32, nnz, "cols")
+        _check_tensor(vals, torch.float32, nnz, "vals")
+        self.device = rows.device
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        need = tsid_workspace_bytes(cfg)
+        self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) & ~255
+        self.cfg = TsidConfig.from_buffer_copy(cfg)
+        self.cfg.stream = self.stream.cuda_stream
+        self.cfg.workspace = base
+        self.cfg.workspace_bytes = need
+        self.m, self.n, self.k, self.nnz = int(cfg.m), int(cfg.n), int(cfg.k), nnz
+        h = C.c_void_p(None)
+        with torch.cuda.device(self.device):
+            st = L.tsid_template_create(C.byref(self.cfg), rows.data_ptr(), cols.data_ptr(), vals.data_ptr(),
+                                        C.byref(h))
+        if st != TSID_OK:
+            self.h = None
+            raise TsidError(st, L.tsid_last_error(None).decode())
+        self.h = h
+
+    # -- the entry points, same names as the header ------------------------------------------------
+    def _raise(self, st):
+        raise TsidError(st, lib().tsid_last_error(self.h).decode())
+
+    def _factors(self, P, Q):
+        _check_tensor(P, torch.float32, self.m * self.k, "P")
+        _check_tensor(Q, torch.float32, self.n * self.k, "Q")
+
+    def tsid_grad_step(self, P, Q, gradP=None, gradQ=None):
+        self._factors(P, Q)
+        if gradP is not None:
+            _check_tensor(gradP, torch.float32, self.m * self.k, "gradP")
+        if gradQ is not None:
+            _check_tensor(gradQ, torch.float32, self.n * self.k, "gradQ")
+        st = lib().tsid_grad_step(self.h, P.data_ptr(), Q.data_ptr(),
+                                  gradP.data_ptr() if gradP is not None else None,
+                                  gradQ.data_ptr() if gradQ is not None else None)
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_fit(self, P, Q, epochs, loss_every=0):
+        self._factors(P, Q)
+        hist = None
+        if loss_every > 0:
+            hist = (C.c_double * (1 + epochs // loss_every))()
+        st = lib().tsid_fit(self.h, P.data_ptr(), Q.data_ptr(), epochs, loss_every, hist)
+        if st != TSID_OK:
+            self._raise(st)
+        return list(hist) if hist is not None else None
+
+    def tsid_loss(self, P, Q):
+        self._factors(P, Q)
+        sse, obj = C.c_double(0), C.c_double(0)
+        st = lib().tsid_loss(self.h, P.data_ptr(), Q.data_ptr(), C.byref(sse), C.byref(obj))
+        if st != TSID_OK:
+            self._raise(st)
+        return sse.value, obj.value
+
+    def tsid_check(self):
+        st = lib().tsid_check(self.h)
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_residuals(self, P, Q, e=None):
+        self._factors(P, Q)
+        if e is None:
+            e = torch.empty(self.nnz, dtype=torch.float32, device=self.device)
+        _check_tensor(e, torch.float32, self.nnz, "e")
+        st = lib().tsid_residuals(self.h, P.data_ptr(), Q.data_ptr(), e.data_ptr())
+        if st != TSID_OK:
+            self._raise(st)
+        return e
+
+    def tsid_get_info(self):
+        p, l = C.c_int32(0), C.c_int32(0)
+        lib().tsid_get_info(self.h, C.byref(p), C.byref(l))
+        return p.value, l.value
+
+    def tsid_get_layout(self):
+        """Copies of the layout arrays as torch tensors (row_ptr, col_idx, val_csr, col_ptr, row_idx,
+        val_csc, perm)."""
+        ptrs = [C.c_void_p(None) for _ in range(7)]
+        st = lib().tsid_get_layout(self.h, *[C.byref(p) for p in ptrs])
+        if st != TSID_OK:
+            self._raise(st)
+        base = (self.workspace.data_ptr() + 255) & ~255
+        spec = [(torch.int64, self.m + 1), (torch.int32, self.nnz), (torch.float32, self.nnz),
+                (torch.int64, self.n + 1), (torch.int32, self.nnz), (torch.float32, self.nnz),
+                (torch.int32, self.nnz)]   # perm is uint32; viewed as int32 (nnz < 2^31)
+        out = []
+        self.stream.synchronize()
+        for p, (dt, cnt) in zip(ptrs, spec):
+            off = p.value - base + (base - self.workspace.data_ptr())
+            nbytes = cnt * torch.empty(0, dtype=dt).element_size()
+            out.append(self.workspace[off:off + nbytes].view(dt).clone())
+        return out
+
+    def tsid_destroy(self):
+        if getattr(self, "h", None) is not None:
+            lib().tsid_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.tsid_destroy()
+        except Exception:
+            pass
+
+
+def template_from_workload(tpl, path=TSID_PATH_AUTO, flags=0, precision=None) -> Template:
+    """Creates a Template from a workloads.Template (device tensors) with its step parameters."""
+    w = tpl.w
+    prec = precision if precision is not None else (TSID_BF16_SHADOW if w.precision == "bf16" else TSID_F32)
+    cfg = make_config(w.m, w.n, w.k, tpl.nnz, prec, path, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q, flags)
+    return Template(cfg, tpl.rows, tpl.cols, tpl.vals)

@@ -1,0 +1,261 @@
+// Host side of the C ABI declared in include/tsid.h: argument checks, workspace carving,
+// and the order of kernel launches of each entry point.  No device allocation happens here.
+#include <new>
+#include <string.h>
+
+#include "tsid_internal.cuh"
+
+using namespace tsid;
+
+namespace {
+
+thread_local char g_create_err[256] = "";
+
+tsid_status_t fail(tsid_template *t, tsid_status_t st, const char *fmt, const char *detail = "") {
+  char *dst = t ? t->err : g_create_err;
+  snprintf(dst, 256, fmt, detail);
+  return st;
+}
+
+tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
+  if (!c) { snprintf(err, 256, "cfg is null"); return TSID_ERR_INVALID_ARG; }
+  if (c->m < 1 || c->n < 1 || c->nnz < 0) { snprintf(err, 256, "m, n must be >= 1 and nnz >= 0"); return TSID_ERR_INVALID_ARG; }
+  if (c->nnz > 2147483647LL) { snprintf(err, 256, "nnz exceeds 2^31-1"); return TSID_ERR_UNSUPPORTED; }
+  if (c->precision != TSID_F32 && c->precision != TSID_BF16_SHADOW) { snprintf(err, 256, "bad precision"); return TSID_ERR_INVALID_ARG; }
+  if (c->path < TSID_PATH_AUTO || c->path > TSID_PATH_DENSE_TC) { snprintf(err, 256, "bad path"); return TSID_ERR_INVALID_ARG; }
+  if (c->clip < TSID_CLIP_NONE || c->clip > TSID_CLIP_ASYM_GRAD) { snprintf(err, 256, "bad clip mode"); return TSID_ERR_INVALID_ARG; }
+  if (c->norm_p < 0 || c->norm_p > 1 || c->norm_q < 0 || c->norm_q > 1) { snprintf(err, 256, "bad norm mode"); return TSID_ERR_INVALID_ARG; }
+  const int mult = c->precision == TSID_BF16_SHADOW ? 8 : 4;
+  if (c->k < 1 || c->k > 256 || c->k % mult) { snprintf(err, 256, "k must be in [1,256] and a multiple of %d", mult); return TSID_ERR_UNSUPPORTED; }
+  if (c->clip != TSID_CLIP_NONE && !(c->xi > 0.f)) { snprintf(err, 256, "xi must be > 0 when clipping"); return TSID_ERR_INVALID_ARG; }
+  return TSID_OK;
+}
+
+int resolve_path(const tsid_config_t &c) {
+  if (c.path != TSID_PATH_AUTO) return c.path;
+  return TSID_PATH_SPARSE;
+}
+
+// Carves (or, with a null base, measures) every device buffer of a template.
+void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScratch &ls) {
+  const size_t nnz = (size_t)c.nnz, m = (size_t)c.m, n = (size_t)c.n, k = (size_t)c.k;
+  const size_t nz = nnz ? nnz : 1;
+  t->flags = cv.take<int32_t>(FLAG_COUNT);
+  t->row_ptr = cv.take<int64_t>(m + 1);
+  t->col_ptr = cv.take<int64_t>(n + 1);
+  t->col_idx = cv.take<int32_t>(nz);
+  t->val_csr = cv.take<float>(nz);
+  t->row_idx = cv.take<int32_t>(nz);
+  t->val_csc = cv.take<float>(nz);
+  t->perm = cv.take<uint32_t>(nz);
+  const size_t per = nnz / kSegLen;
+  Side *sides[2] = {&t->rowside, &t->colside};
+  for (int i = 0; i < 2; ++i) {
+    Side &sd = *sides[i];
+    sd.nrows = (int32_t)(i == 0 ? m : n);
+    sd.cap_seg = (int32_t)(sd.nrows + per + 1);
+    sd.cap_split = (int32_t)(per + 1);
+    sd.cap_slot = (int32_t)(2 * per + 2);
+    sd.segs = cv.take<Segment>(sd.cap_seg);
+    sd.splits = cv.take<SplitRow>(sd.cap_split);
+    sd.scale = cv.take<float>(sd.nrows);
+    sd.G = cv.take<float>((size_t)sd.nrows * k);
+    sd.shadow = c.precision == TSID_BF16_SHADOW ? cv.take<__nv_bfloat16>((size_t)sd.nrows * k) : nullptr;
+  }
+  t->rowside.ptr = t->row_ptr; t->rowside.idx = t->col_idx; t->rowside.val = t->val_csr;
+  t->colside.ptr = t->col_ptr; t->colside.idx = t->row_idx; t->colside.val = t->val_csc;
+  t->partial = cv.take<float>((2 * per + 2) * k);
+  t->red_cap = (int32_t)(2 + 2 * 256 + t->rowside.cap_seg);
+  t->red = cv.take<double>(t->red_cap);
+  // transient buffers of the layout pass
+  ls.kA = cv.take<uint32_t>(nz); ls.kB = cv.take<uint32_t>(nz);
+  ls.vA = cv.take<uint32_t>(nz); ls.vB = cv.take<uint32_t>(nz);
+  ls.hist = cv.take<uint32_t>(256 * (size_t)kSortBlocksMax);
+  const size_t mx = (m > n ? m : n) + 2;
+  ls.scanA = cv.take<uint32_t>(mx); ls.scanB = cv.take<uint32_t>(mx); ls.scanC = cv.take<uint32_t>(mx);
+  ls.blocksums = cv.take<uint32_t>(kScanBlocksMax);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+tsid_status_t cuda_fail(tsid_template *t, cudaError_t e) {
+  return fail(t, TSID_ERR_CUDA, "CUDA error: %s", cudaGetErrorString(e));
+}
+
+tsid_status_t check_factors(tsid_template *t, const float *P, const float *Q) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (!P || !Q) return fail(t, TSID_ERR_INVALID_ARG, "P or Q is null");
+  if (!aligned16(P) || !aligned16(Q)) return fail(t, TSID_ERR_INVALID_ARG, "P and Q must be 16-byte aligned");
+  return TSID_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+tsid_status_t tsid_workspace_bytes(const tsid_config_t *cfg, size_t *h_bytes_out) {
+  if (!h_bytes_out) return fail(nullptr, TSID_ERR_INVALID_ARG, "bytes_out is null");
+  tsid_status_t st = check_cfg(cfg, g_create_err);
+  if (st != TSID_OK) return st;
+  tsid_template tmp;
+  memset(static_cast<void *>(&tmp), 0, sizeof(tmp));
+  Carver cv(nullptr);
+  LayoutScratch ls;
+  carve_all(&tmp, *cfg, cv, ls);
+  *h_bytes_out = cv.off;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_rows, const int32_t *d_cols,
+                                   const float *d_vals, tsid_template_t **out) {
+  if (!out) return fail(nullptr, TSID_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  tsid_status_t st = check_cfg(cfg, g_create_err);
+  if (st != TSID_OK) return st;
+  if (cfg->nnz > 0 && (!d_rows || !d_cols || !d_vals)) return fail(nullptr, TSID_ERR_INVALID_ARG, "COO pointer is null");
+  if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255u))
+    return fail(nullptr, TSID_ERR_INVALID_ARG, "workspace is null or not 256-byte aligned");
+  size_t need = 0;
+  tsid_workspace_bytes(cfg, &need);
+  if (cfg->workspace_bytes < need) return fail(nullptr, TSID_ERR_OOM, "workspace smaller than tsid_workspace_bytes");
+  const int path = resolve_path(*cfg);
+  if (path == TSID_PATH_DENSE_TC) return fail(nullptr, TSID_ERR_UNSUPPORTED, "dense tensor-core path not available for this template");
+
+  tsid_template *t = new (std::nothrow) tsid_template;
+  if (!t) return fail(nullptr, TSID_ERR_OOM, "host allocation failed");
+  memset(static_cast<void *>(t), 0, sizeof(*t));
+  t->cfg = *cfg;
+  t->stream = static_cast<cudaStream_t>(cfg->stream);
+  t->path = path;
+  Carver cv(cfg->workspace);
+  LayoutScratch ls;
+  carve_all(t, *cfg, cv, ls);
+
+  int32_t hf[FLAG_COUNT] = {0};
+  cudaError_t e = layout_build(t, d_rows, d_cols, d_vals, ls, hf);
+  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); delete t; return st; }
+  if (hf[FLAG_RANGE]) { delete t; return fail(nullptr, TSID_ERR_INDEX_RANGE, "a row or column index is out of range"); }
+  if (hf[FLAG_UNSORTED] && (cfg->flags & TSID_INPUT_ROW_SORTED)) { delete t; return fail(nullptr, TSID_ERR_UNSORTED, "input promised row-sorted but is not"); }
+  if (hf[FLAG_DUP] && (cfg->flags & TSID_VALIDATE)) { delete t; return fail(nullptr, TSID_ERR_DUPLICATE, "duplicate (row, col) in Omega"); }
+  e = build_segments(t, t->rowside, cfg->norm_p, ls);
+  if (e == cudaSuccess) e = build_segments(t, t->colside, cfg->norm_q, ls);
+  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); delete t; return st; }
+  snprintf(t->err, 256, "ok");
+  *out = t;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *d_gradP_or_null,
+                             float *d_gradQ_or_null) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  if ((d_gradP_or_null && !aligned16(d_gradP_or_null)) || (d_gradQ_or_null && !aligned16(d_gradQ_or_null)))
+    return fail(t, TSID_ERR_INVALID_ARG, "gradient outputs must be 16-byte aligned");
+  float *GP = d_gradP_or_null ? d_gradP_or_null : t->rowside.G;
+  float *GQ = d_gradQ_or_null ? d_gradQ_or_null : t->colside.G;
+  cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
+  if (e == cudaSuccess) e = sparse_grad(t, d_P, d_Q, GP, GQ);
+  if (e == cudaSuccess) e = sparse_update(t, d_P, d_Q, GP, GQ);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+static tsid_status_t loss_sync(tsid_template *t, const float *d_P, const float *d_Q, double *sse, double *sq) {
+  cudaError_t e = sparse_loss(t, d_P, d_Q, t->red);
+  double h[2] = {0, 0};
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h, t->red, 2 * sizeof(double), cudaMemcpyDeviceToHost, t->stream);
+  int32_t hf[FLAG_COUNT] = {0};
+  if (e == cudaSuccess) e = cudaMemcpyAsync(hf, t->flags, sizeof(hf), cudaMemcpyDeviceToHost, t->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
+  if (e != cudaSuccess) return cuda_fail(t, e);
+  *sse = h[0];
+  *sq = h[1];
+  if (hf[FLAG_NONFINITE] || !(h[0] == h[0]) || !(h[1] == h[1]))
+    return fail(t, TSID_ERR_NONFINITE, "a factor became non-finite");
+  return TSID_OK;
+}
+
+tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epochs, int32_t loss_every,
+                       double *h_sse_history_or_null) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  if (epochs < 0 || loss_every < 0) return fail(t, TSID_ERR_INVALID_ARG, "epochs and loss_every must be >= 0");
+  int nh = 0;
+  double sse, sq;
+  if (loss_every > 0) {
+    st = loss_sync(t, d_P, d_Q, &sse, &sq);
+    if (h_sse_history_or_null) h_sse_history_or_null[nh] = sse;
+    ++nh;
+    if (st != TSID_OK) return st;
+  }
+  cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
+  for (int ep = 0; ep < epochs && e == cudaSuccess; ++ep) {
+    // the update kernel refreshes the shadows, so they stay current between epochs
+    e = sparse_grad(t, d_P, d_Q, t->rowside.G, t->colside.G);
+    if (e == cudaSuccess) e = sparse_update(t, d_P, d_Q, t->rowside.G, t->colside.G);
+    if (e == cudaSuccess && loss_every > 0 && (ep + 1) % loss_every == 0) {
+      st = loss_sync(t, d_P, d_Q, &sse, &sq);
+      if (h_sse_history_or_null) h_sse_history_or_null[nh] = sse;
+      ++nh;
+      if (st != TSID_OK) return st;
+    }
+  }
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+tsid_status_t tsid_loss(tsid_template_t *t, const float *d_P, const float *d_Q, double *h_sse, double *h_objective) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  double sse = 0, sq = 0;
+  st = loss_sync(t, d_P, d_Q, &sse, &sq);
+  if (h_sse) *h_sse = sse;
+  if (h_objective) *h_objective = sse + (double)t->cfg.lambda * sq;
+  return st;
+}
+
+tsid_status_t tsid_check(tsid_template_t *t) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  int32_t hf[FLAG_COUNT] = {0};
+  cudaError_t e = cudaMemcpyAsync(hf, t->flags, sizeof(hf), cudaMemcpyDeviceToHost, t->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
+  if (e != cudaSuccess) return cuda_fail(t, e);
+  if (hf[FLAG_NONFINITE]) return fail(t, TSID_ERR_NONFINITE, "a factor became non-finite");
+  return TSID_OK;
+}
+
+tsid_status_t tsid_destroy(tsid_template_t *t) {
+  delete t;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_get_layout(tsid_template_t *t, const int64_t **d_row_ptr, const int32_t **d_col_idx,
+                              const float **d_val_csr, const int64_t **d_col_ptr, const int32_t **d_row_idx,
+                              const float **d_val_csc, const uint32_t **d_perm) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (d_row_ptr) *d_row_ptr = t->row_ptr;
+  if (d_col_idx) *d_col_idx = t->col_idx;
+  if (d_val_csr) *d_val_csr = t->val_csr;
+  if (d_col_ptr) *d_col_ptr = t->col_ptr;
+  if (d_row_idx) *d_row_idx = t->row_idx;
+  if (d_val_csc) *d_val_csc = t->val_csc;
+  if (d_perm) *d_perm = t->perm;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *d_Q, float *d_e_csr) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  if (!d_e_csr && t->cfg.nnz > 0) return fail(t, TSID_ERR_INVALID_ARG, "e output is null");
+  cudaError_t e = sparse_residuals(t, d_P, d_Q, d_e_csr);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (h_path) *h_path = t->path;
+  if (h_launches_per_step) *h_launches_per_step = sparse_launches_per_step(t);
+  return TSID_OK;
+}
+
+const char *tsid_last_error(const tsid_template_t *t) { return t ? t->err : g_create_err; }
+
+}  // extern "C"

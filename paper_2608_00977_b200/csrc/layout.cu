@@ -1,0 +1,421 @@
+// Layout pass: COO -> CSR sorted by (row, col), CSC sorted by (col, row), perm, and the
+// equal-length work segments of the two gather-reduce passes.  Integer work only; every
+// output is unique (stable sorts), so it can be compared bit for bit with a CPU sort.
+//
+// The sort is a hand-written stable LSD radix sort of (uint32 key, uint32 payload) pairs:
+// per pass a per-block digit histogram, an exclusive scan over the (digit, block) matrix and
+// a scatter that ranks the items of each tile in input order (warp match + per-warp digit
+// counters).  Integer atomics appear only in shared-memory histograms; nothing here
+// depends on their order.
+#include "tsid_internal.cuh"
+
+namespace tsid {
+
+namespace {
+
+constexpr int RS_THREADS = 256;
+constexpr int RS_WARPS = RS_THREADS / 32;
+constexpr int RS_ITEMS = 8;
+constexpr int RS_TILE = RS_THREADS * RS_ITEMS;  // 2048 pairs per tile
+constexpr int RS_RADIX = 256;
+
+#define CK(x)                        \
+  do {                               \
+    cudaError_t e_ = (x);            \
+    if (e_ != cudaSuccess) return e_; \
+  } while (0)
+
+// ---- radix sort ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(RS_THREADS)
+rs_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int64_t per_block, int shift,
+               uint32_t mask, uint32_t *__restrict__ hist, int nb) {
+  __shared__ uint32_t h[RS_RADIX];
+  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) h[d] = 0;
+  __syncthreads();
+  int64_t lo = (int64_t)blockIdx.x * per_block;
+  int64_t hi = lo + per_block < n ? lo + per_block : n;
+  for (int64_t p = lo + threadIdx.x; p < hi; p += RS_THREADS)
+    atomicAdd(&h[(keys[p] >> shift) & mask], 1u);
+  __syncthreads();
+  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) hist[(size_t)d * nb + blockIdx.x] = h[d];
+}
+
+// Exclusive scan of a short array (<= 256 * kSortBlocksMax) by one block.
+__global__ void __launch_bounds__(1024) rs_scan_kernel(uint32_t *a, int n) {
+  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t carry_s;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  for (int base = 0; base < n; base += 1024) {
+    int i = base + threadIdx.x;
+    uint32_t v = i < n ? a[i] : 0u;
+    uint32_t inc = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += u;
+    }
+    if (lane == 31) warp_tot[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+      uint32_t t = warp_tot[lane];
+      uint32_t ti = t;
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t u = __shfl_up_sync(0xffffffffu, ti, o);
+        if (lane >= o) ti += u;
+      }
+      warp_tot[lane] = ti - t;  // exclusive prefix of the warp totals
+    }
+    __syncthreads();
+    uint32_t carry = carry_s;
+    uint32_t excl = carry + warp_tot[w] + inc - v;
+    if (i < n) a[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry_s = excl + v;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(RS_THREADS)
+rs_scatter_kernel(const uint32_t *__restrict__ kin, const uint32_t *__restrict__ vin,
+                  uint32_t *__restrict__ kout, uint32_t *__restrict__ vout, int64_t n,
+                  int64_t per_block, int shift, uint32_t mask, const uint32_t *__restrict__ offs,
+                  int nb) {
+  __shared__ uint32_t wc[RS_WARPS][RS_RADIX];
+  __shared__ uint32_t off[RS_RADIX];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
+  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) off[d] = offs[(size_t)d * nb + blockIdx.x];
+  int64_t lo = (int64_t)blockIdx.x * per_block;
+  int64_t hi = lo + per_block < n ? lo + per_block : n;
+  for (int64_t tile = lo; tile < hi; tile += RS_TILE) {
+    for (int d = lane; d < RS_RADIX; d += 32) wc[w][d] = 0;
+    __syncthreads();  // also orders the initial off[] load and the previous tile's reads
+    uint32_t key[RS_ITEMS], val[RS_ITEMS], rank[RS_ITEMS], dig[RS_ITEMS];
+    const int64_t wbase = tile + (int64_t)w * 32 * RS_ITEMS;
+#pragma unroll
+    for (int it = 0; it < RS_ITEMS; ++it) {
+      int64_t p = wbase + it * 32 + lane;
+      bool ok = p < hi;
+      key[it] = ok ? kin[p] : 0u;
+      val[it] = ok ? (vin ? vin[p] : (uint32_t)p) : 0u;
+      dig[it] = ok ? ((key[it] >> shift) & mask) : 0xffffffffu;
+    }
+#pragma unroll
+    for (int it = 0; it < RS_ITEMS; ++it) {
+      uint32_t peers = __match_any_sync(0xffffffffu, dig[it]);
+      int leader = __ffs(peers) - 1;
+      uint32_t base = 0;
+      if (lane == leader && dig[it] != 0xffffffffu) {
+        base = wc[w][dig[it]];
+        wc[w][dig[it]] = base + __popc(peers);
+      }
+      base = __shfl_sync(0xffffffffu, base, leader);
+      rank[it] = base + __popc(peers & lt);
+      __syncwarp();
+    }
+    __syncthreads();
+    {  // thread d: exclusive scan of digit d over the warps, shifted by the running offset
+      int d = threadIdx.x;
+      uint32_t run = off[d];
+#pragma unroll
+      for (int ww = 0; ww < RS_WARPS; ++ww) {
+        uint32_t c = wc[ww][d];
+        wc[ww][d] = run;
+        run += c;
+      }
+      off[d] = run;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < RS_ITEMS; ++it) {
+      if (dig[it] != 0xffffffffu) {
+        uint32_t pos = wc[w][dig[it]] + rank[it];
+        kout[pos] = key[it];
+        vout[pos] = val[it];
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Stable sort of n pairs on key bits [0, nbits).  Reads (kin, vin) (vin == nullptr: the
+// payload is the position), ping-pongs between (kA, vA) and (kB, vB); *kres / *vres point at
+// the buffers holding the result.
+cudaError_t radix_sort_pairs(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits,
+                             LayoutScratch &s, cudaStream_t st, uint32_t **kres, uint32_t **vres) {
+  int npass = (nbits + 7) / 8;
+  if (npass < 1) npass = 1;
+  int64_t tiles = (n + RS_TILE - 1) / RS_TILE;
+  int nb = (int)(tiles < kSortBlocksMax ? tiles : kSortBlocksMax);
+  if (nb < 1) nb = 1;
+  int64_t per_block = ((tiles + nb - 1) / nb) * RS_TILE;
+  const uint32_t *ck = kin, *cv = vin;
+  uint32_t *ok = s.kA, *ov = s.vA;
+  int shift = 0;
+  for (int p = 0; p < npass; ++p) {
+    int bits = (nbits - shift + (npass - p) - 1) / (npass - p);  // spread the bits evenly
+    if (bits < 1) bits = 1;
+    uint32_t mask = (1u << bits) - 1u;
+    rs_hist_kernel<<<nb, RS_THREADS, 0, st>>>(ck, n, per_block, shift, mask, s.hist, nb);
+    rs_scan_kernel<<<1, 1024, 0, st>>>(s.hist, RS_RADIX * nb);
+    rs_scatter_kernel<<<nb, RS_THREADS, 0, st>>>(ck, cv, ok, ov, n, per_block, shift, mask, s.hist, nb);
+    CK(cudaGetLastError());
+    ck = ok; cv = ov;
+    if (ok == s.kA) { ok = s.kB; ov = s.vB; } else { ok = s.kA; ov = s.vA; }
+    shift += bits;
+  }
+  *kres = const_cast<uint32_t *>(ck);
+  *vres = const_cast<uint32_t *>(cv);
+  return cudaSuccess;
+}
+
+// ---- generic exclusive scan of uint32 (three kernels; block sums scanned by one block) -----
+constexpr int SC_THREADS = 256, SC_ITEMS = 8, SC_TILE = SC_THREADS * SC_ITEMS;
+
+__global__ void __launch_bounds__(SC_THREADS)
+scan_tile_kernel(const uint32_t *in, uint32_t *out, int64_t n,  // in may alias out
+                 uint32_t *__restrict__ blocksums, const uint32_t *__restrict__ blockoffs) {
+  __shared__ uint32_t wt[SC_THREADS / 32];
+  int64_t base = (int64_t)blockIdx.x * SC_TILE + (int64_t)threadIdx.x * SC_ITEMS;
+  uint32_t v[SC_ITEMS], sum = 0;
+#pragma unroll
+  for (int i = 0; i < SC_ITEMS; ++i) {
+    v[i] = (base + i < n) ? in[base + i] : 0u;
+    sum += v[i];
+  }
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  uint32_t inc = sum;
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += u;
+  }
+  if (lane == 31) wt[w] = inc;
+  __syncthreads();
+  uint32_t woff = 0;
+  for (int ww = 0; ww < w; ++ww) woff += wt[ww];
+  if (blockoffs == nullptr) {  // first sweep: only the block total is needed
+    if (threadIdx.x == SC_THREADS - 1) blocksums[blockIdx.x] = woff + inc;
+    return;
+  }
+  uint32_t run = blockoffs[blockIdx.x] + woff + inc - sum;
+#pragma unroll
+  for (int i = 0; i < SC_ITEMS; ++i) {
+    if (base + i < n) out[base + i] = run;
+    run += v[i];
+  }
+}
+
+// out[0..n) = exclusive scan of in[0..n); out[n] = total.  in and out may alias.
+cudaError_t exclusive_scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch &s,
+                               cudaStream_t st) {
+  int64_t n1 = n + 1;  // scan n+1 slots so that out[n] receives the total (in[n] must be 0)
+  int nb = (int)((n1 + SC_TILE - 1) / SC_TILE);
+  if (nb > kScanBlocksMax) return cudaErrorInvalidValue;
+  scan_tile_kernel<<<nb, SC_THREADS, 0, st>>>(in, nullptr, n1, s.blocksums, nullptr);
+  rs_scan_kernel<<<1, 1024, 0, st>>>(s.blocksums, nb);
+  scan_tile_kernel<<<nb, SC_THREADS, 0, st>>>(in, out, n1, nullptr, s.blocksums);
+  return cudaGetLastError();
+}
+
+// ---- checks, gathers, pointer arrays ------------------------------------------------------------
+__global__ void check_coo_kernel(const int32_t *__restrict__ rows, const int32_t *__restrict__ cols,
+                                 int64_t nnz, int32_t m, int32_t n, int32_t *flags) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  bool bad = false, unsorted = false, dup = false;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nnz; t += stride) {
+    int32_t r = rows[t], c = cols[t];
+    if (r < 0 || r >= m || c < 0 || c >= n) bad = true;
+    if (t > 0) {
+      int32_t r0 = rows[t - 1], c0 = cols[t - 1];
+      if (r0 > r || (r0 == r && c0 > c)) unsorted = true;
+      if (r0 == r && c0 == c) dup = true;
+    }
+  }
+  if (bad) flags[FLAG_RANGE] = 1;
+  if (unsorted) flags[FLAG_UNSORTED] = 1;
+  if (dup) flags[FLAG_DUP] = 1;  // only meaningful when the input is sorted
+}
+
+__global__ void check_dup_kernel(const uint32_t *__restrict__ rowkey, const int32_t *__restrict__ col_idx,
+                                 int64_t nnz, int32_t *flags) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  bool dup = false;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x + 1; p < nnz; p += stride)
+    if (rowkey[p] == rowkey[p - 1] && col_idx[p] == col_idx[p - 1]) dup = true;
+  if (dup) flags[FLAG_DUP] = 1;
+}
+
+template <typename TI, typename TO>
+__global__ void gather_kernel(const TI *__restrict__ src, const uint32_t *__restrict__ pos, TO *__restrict__ dst,
+                              int64_t n) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += stride)
+    dst[p] = (TO)src[pos[p]];
+}
+
+template <typename TI, typename TO>
+__global__ void copy_kernel(const TI *__restrict__ src, TO *__restrict__ dst, int64_t n) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += stride) dst[p] = (TO)src[p];
+}
+
+// ptr[r] = first position p with key[p] >= r, for r in [0, nrows]; keys are sorted.
+__global__ void ptr_from_sorted_kernel(const uint32_t *__restrict__ key, int64_t nnz, int32_t nrows,
+                                       int64_t *__restrict__ ptr) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p <= nnz; p += stride) {
+    int64_t lo = (p == 0) ? 0 : (int64_t)key[p - 1] + 1;       // rows (key[p-1], key[p]] start at p
+    int64_t hi = (p == nnz) ? (int64_t)nrows : (int64_t)key[p];
+    for (int64_t r = lo; r <= hi; ++r) ptr[r] = p;
+  }
+}
+
+// ---- segments ---------------------------------------------------------------------------------------
+__global__ void seg_count_kernel(const int64_t *__restrict__ ptr, int32_t nrows, int norm_count,
+                                 uint32_t *__restrict__ nseg, uint32_t *__restrict__ nslot,
+                                 uint32_t *__restrict__ nsplit, float *__restrict__ scale) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i <= nrows; i += stride) {
+    if (i == nrows) { nseg[i] = 0; nslot[i] = 0; nsplit[i] = 0; continue; }
+    int64_t cnt = ptr[i + 1] - ptr[i];
+    uint32_t s = cnt <= kSegLen ? 1u : (uint32_t)((cnt + kSegLen - 1) / kSegLen);
+    nseg[i] = s;
+    nslot[i] = s > 1 ? s : 0u;
+    nsplit[i] = s > 1 ? 1u : 0u;
+    float sc = (norm_count && cnt > 1) ? (float)cnt : 1.0f;
+    scale[i] = 2.0f / sc;
+  }
+}
+
+__global__ void seg_fill_kernel(const int64_t *__restrict__ ptr, int32_t nrows,
+                                const uint32_t *__restrict__ seg_off, const uint32_t *__restrict__ slot_off,
+                                const uint32_t *__restrict__ split_off, Segment *__restrict__ segs,
+                                SplitRow *__restrict__ splits) {
+  // one warp per row: the lanes stride over the row's segments
+  int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int lane = threadIdx.x & 31;
+  int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t i = warp; i < nrows; i += nwarps) {
+    int64_t b = ptr[i], cnt = ptr[i + 1] - b;
+    uint32_t s0 = seg_off[i], ns = seg_off[i + 1] - s0;
+    bool split = ns > 1;
+    uint32_t sl0 = slot_off[i];
+    for (uint32_t q = lane; q < ns; q += 32) {
+      Segment sg;
+      sg.row = (int32_t)i;
+      sg.begin = (uint32_t)(b + (int64_t)q * kSegLen);
+      int64_t rem = cnt - (int64_t)q * kSegLen;
+      sg.len = (int32_t)(rem < kSegLen ? rem : kSegLen);
+      sg.slot = split ? (int32_t)(sl0 + q) : -1;
+      segs[s0 + q] = sg;
+    }
+    if (split && lane == 0) {
+      SplitRow sr;
+      sr.row = (int32_t)i; sr.slot0 = (int32_t)sl0; sr.nseg = (int32_t)ns; sr.pad = 0;
+      splits[split_off[i]] = sr;
+    }
+  }
+}
+
+inline int grid_for(int64_t n, int threads) {
+  int64_t g = (n + threads - 1) / threads;
+  if (g < 1) g = 1;
+  if (g > 148 * 16) g = 148 * 16;
+  return (int)g;
+}
+
+}  // namespace
+
+cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols,
+                         const float *d_vals, LayoutScratch &s, int32_t h_flags[FLAG_COUNT]) {
+  cudaStream_t st = t->stream;
+  const int64_t nnz = t->cfg.nnz;
+  const int32_t m = t->cfg.m, n = t->cfg.n;
+  CK(cudaMemsetAsync(t->flags, 0, sizeof(int32_t) * FLAG_COUNT, st));
+  if (nnz > 0) check_coo_kernel<<<grid_for(nnz, 256), 256, 0, st>>>(d_rows, d_cols, nnz, m, n, t->flags);
+  CK(cudaGetLastError());
+  CK(cudaMemcpyAsync(h_flags, t->flags, sizeof(int32_t) * FLAG_COUNT, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  if (h_flags[FLAG_RANGE]) return cudaSuccess;  // caller reports TSID_ERR_INDEX_RANGE
+  if (h_flags[FLAG_UNSORTED] && (t->cfg.flags & TSID_INPUT_ROW_SORTED)) return cudaSuccess;
+
+  const int g = grid_for(nnz, 256);
+  uint32_t *rowkey = reinterpret_cast<uint32_t *>(t->val_csc);  // parked here until val_csc is written
+  if (nnz > 0) {
+    if (!h_flags[FLAG_UNSORTED]) {
+      // already in (row, col) order: CSR is the input
+      copy_kernel<int32_t, int32_t><<<g, 256, 0, st>>>(d_cols, t->col_idx, nnz);
+      copy_kernel<float, float><<<g, 256, 0, st>>>(d_vals, t->val_csr, nnz);
+      copy_kernel<int32_t, uint32_t><<<g, 256, 0, st>>>(d_rows, rowkey, nnz);
+    } else {
+      h_flags[FLAG_DUP] = 0;  // the adjacent-pair test of check_coo only holds for sorted input
+      CK(cudaMemsetAsync(t->flags + FLAG_DUP, 0, sizeof(int32_t), st));
+      uint32_t *k1, *v1, *k2, *v2;
+      // stable by column, then stable by row  =>  (row, col, input position) order
+      CK(radix_sort_pairs(reinterpret_cast<const uint32_t *>(d_cols), nullptr, nnz, bits_for(n - 1), s, st, &k1, &v1));
+      // keys for the second sort: row of each entry in the current order
+      // (the sort first writes to (kA, vA), so its input must sit in the B buffers; the sorted
+      // column keys in k1 are no longer needed)
+      (void)k1;
+      uint32_t *gk = s.kB;
+      gather_kernel<int32_t, uint32_t><<<g, 256, 0, st>>>(d_rows, v1, gk, nnz);
+      if (v1 == s.vA) { copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(v1, s.vB, nnz); v1 = s.vB; }
+      CK(radix_sort_pairs(gk, v1, nnz, bits_for(m - 1), s, st, &k2, &v2));
+      gather_kernel<int32_t, int32_t><<<g, 256, 0, st>>>(d_cols, v2, t->col_idx, nnz);
+      gather_kernel<float, float><<<g, 256, 0, st>>>(d_vals, v2, t->val_csr, nnz);
+      copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(k2, rowkey, nnz);
+      if (t->cfg.flags & TSID_VALIDATE) check_dup_kernel<<<g, 256, 0, st>>>(rowkey, t->col_idx, nnz, t->flags);
+    }
+    CK(cudaGetLastError());
+  }
+  ptr_from_sorted_kernel<<<grid_for(nnz + 1, 256), 256, 0, st>>>(rowkey, nnz, m, t->row_ptr);
+  CK(cudaGetLastError());
+
+  // CSC: stable sort of the CSR positions by column
+  if (nnz > 0) {
+    uint32_t *k3, *v3;
+    CK(radix_sort_pairs(reinterpret_cast<const uint32_t *>(t->col_idx), nullptr, nnz, bits_for(n - 1), s, st, &k3, &v3));
+    copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(v3, t->perm, nnz);
+    ptr_from_sorted_kernel<<<grid_for(nnz + 1, 256), 256, 0, st>>>(k3, nnz, n, t->col_ptr);
+    gather_kernel<uint32_t, int32_t><<<g, 256, 0, st>>>(rowkey, t->perm, t->row_idx, nnz);
+    gather_kernel<float, float><<<g, 256, 0, st>>>(t->val_csr, t->perm, t->val_csc, nnz);  // overwrites rowkey
+    CK(cudaGetLastError());
+  } else {
+    ptr_from_sorted_kernel<<<1, 256, 0, st>>>(nullptr, 0, n, t->col_ptr);
+    CK(cudaGetLastError());
+  }
+  int32_t dupflag = 0;
+  CK(cudaMemcpyAsync(&dupflag, t->flags + FLAG_DUP, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  h_flags[FLAG_DUP] = dupflag;
+  return cudaSuccess;
+}
+
+cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutScratch &s) {
+  cudaStream_t st = t->stream;
+  const int32_t nr = side.nrows;
+  seg_count_kernel<<<grid_for((int64_t)nr + 1, 256), 256, 0, st>>>(side.ptr, nr, norm_mode == TSID_NORM_COUNT,
+                                                                 s.scanA, s.scanB, s.scanC, side.scale);
+  CK(cudaGetLastError());
+  CK(exclusive_scan_u32(s.scanA, s.scanA, nr, s, st));
+  CK(exclusive_scan_u32(s.scanB, s.scanB, nr, s, st));
+  CK(exclusive_scan_u32(s.scanC, s.scanC, nr, s, st));
+  uint32_t tot[3];
+  CK(cudaMemcpyAsync(&tot[0], s.scanA + nr, 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(&tot[1], s.scanB + nr, 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(&tot[2], s.scanC + nr, 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  side.nseg = (int32_t)tot[0];
+  side.nslot = (int32_t)tot[1];
+  side.nsplit = (int32_t)tot[2];
+  if (side.nseg > side.cap_seg || side.nslot > side.cap_slot || side.nsplit > side.cap_split)
+    return cudaErrorMemoryAllocation;
+  int64_t threads = (int64_t)nr * 32;
+  seg_fill_kernel<<<grid_for(threads, 256), 256, 0, st>>>(side.ptr, nr, s.scanA, s.scanB, s.scanC, side.segs,
+                                                         side.splits);
+  CK(cudaGetLastError());
+  return cudaStreamSynchronize(st);
+}
+
+}  // namespace tsid

@@ -1,0 +1,120 @@
+// Internal declarations shared by the translation units of libtsid (host side of the
+// C ABI, layout pass, sparse passes, dense tensor-core variant).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "../../include/tsid.h"
+
+namespace tsid {
+
+// Longest run of entries one warp reduces in registers before the result goes through the
+// grid-level (fixed order) reduction.  Also the unit of load balance under skewed degrees.
+constexpr int kSegLen = 1024;
+
+// One unit of work of a gather-reduce pass: `len` consecutive entries of one row (CSR pass)
+// or one column (CSC pass).  slot < 0: the row has a single segment and the warp writes the
+// gradient row directly; slot >= 0: index of the partial row the fix-up kernel sums later.
+struct __align__(16) Segment {
+  int32_t row;
+  uint32_t begin;
+  int32_t len;
+  int32_t slot;
+};
+
+// A row (column) that spans several segments: partial rows [slot0, slot0 + nseg).
+struct __align__(16) SplitRow {
+  int32_t row;
+  int32_t slot0;
+  int32_t nseg;
+  int32_t pad;
+};
+
+// One side (rows for the CSR pass, columns for the CSC pass).
+struct Side {
+  int32_t nrows = 0;       // m or n
+  const int64_t *ptr = nullptr;   // [nrows+1]
+  const int32_t *idx = nullptr;   // [nnz] opposite-side index of each entry
+  const float *val = nullptr;     // [nnz]
+  Segment *segs = nullptr;
+  SplitRow *splits = nullptr;
+  float *scale = nullptr;  // [nrows] 2 / s_i
+  float *G = nullptr;      // [nrows * k] internal gradient buffer
+  __nv_bfloat16 *shadow = nullptr;  // [nrows * k] or null
+  int32_t nseg = 0, nsplit = 0, nslot = 0;
+  int32_t cap_seg = 0, cap_split = 0, cap_slot = 0;
+};
+
+struct DenseState;  // dense_tc.cu
+
+}  // namespace tsid
+
+struct tsid_template {
+  tsid_config_t cfg;
+  cudaStream_t stream;
+  int path;  // resolved tsid_path_t
+  tsid::Side rowside, colside;
+  // layout arrays (device, in the workspace)
+  int64_t *row_ptr, *col_ptr;
+  int32_t *col_idx, *row_idx;
+  float *val_csr, *val_csc;
+  uint32_t *perm;
+  float *partial;     // [max(nslot_row, nslot_col) * k]
+  double *red;        // reduction scratch for the loss
+  int32_t red_cap;
+  int32_t *flags;     // device flags: [0] range, [1] unsorted, [2] duplicate, [3] non-finite
+  tsid::DenseState *dense;
+  char err[256];
+};
+
+namespace tsid {
+
+enum { FLAG_RANGE = 0, FLAG_UNSORTED = 1, FLAG_DUP = 2, FLAG_NONFINITE = 3, FLAG_COUNT = 8 };
+
+// Carves 256-byte aligned pieces out of the caller's workspace; with base == nullptr it
+// only measures.
+struct Carver {
+  char *base;
+  size_t off = 0;
+  explicit Carver(void *b) : base(static_cast<char *>(b)) {}
+  template <typename T>
+  T *take(size_t count) {
+    size_t bytes = (count * sizeof(T) + 255) & ~size_t(255);
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+// Transient buffers of the layout pass (also carved from the workspace).
+struct LayoutScratch {
+  uint32_t *kA, *kB, *vA, *vB;  // [nnz] each
+  uint32_t *hist;               // [256 * kSortBlocks]
+  uint32_t *scanA, *scanB, *scanC;  // [max(m,n)+1] each
+  uint32_t *blocksums;          // [kScanBlocksMax]
+};
+constexpr int kSortBlocksMax = 2048;
+constexpr int kScanBlocksMax = 1 << 20;
+
+cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols,
+                         const float *d_vals, LayoutScratch &s, int32_t h_flags[FLAG_COUNT]);
+cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutScratch &s);
+
+// sparse passes (sparse.cu)
+cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);
+cudaError_t sparse_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ);
+cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ);
+cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_Q, float *d_e);
+cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
+int sparse_launches_per_step(const tsid_template *t);
+
+inline int bits_for(uint32_t maxval) {  // number of bits needed to represent values <= maxval
+  int b = 0;
+  while (b < 32 && (maxval >> b) != 0) ++b;
+  return b < 1 ? 1 : b;
+}
+
+}  // namespace tsid
