@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the template-recovery hot path: observed-entry gradient updates per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C5] [--impl reference]
+
+A step is one full-batch tsid_grad_step (row pass, column pass, fix-ups, clip + update; for
+bf16 templates also the shadow refresh) over the whole synthetic template, inputs resident in
+HBM.  One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs an independent
+replica of the same template (the path is single-GPU; there is no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "observed-entry gradient updates/sec"
+UNIT = "updates/s"
+L2_BYTES = 126 * 1024 * 1024
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gather-reduce pass kernel
+# (average of the row pass and the column pass), from the ncu summaries under profiles/.
+NCU_TRAFFIC_PER_LAUNCH = {
+    "C5": 91.79e9,   # profiles/pass_kernel_C5_launches_dram.md: row 76.95 GB, column 106.63 GB
+    "C3": 0.882e9,   # profiles/pass_kernel_C3_ncu_full.md: row 0.892 GB, column 0.872 GB
+}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def alg_bytes(w, nnz, nseg_row, nseg_col):
+    """Algorithmic bytes of one launch of each kernel of a step ("Roofline")."""
+    b = 2 if w.precision == "bf16" else 4
+    k = w.k
+    row = nnz * (8 + k * b) + w.m * k * (b + 4) + nseg_row * 16
+    col = nnz * (8 + k * b) + w.n * k * (b + 4) + nseg_col * 16
+    upd = (w.m + w.n) * k * (4 + 4 + 4 + (b if b == 2 else 0)) + (w.m + w.n) * 4
+    return row, col, upd
+
+
+def run_reference(args, W):
+    """The oracle, as it stands, on the host cores: each step is one oracle step over a bounded
+    sample (a prefix of the row-sorted COO) of the workload."""
+    import numpy as np
+    import oracle
+    w = W.CONFIGS[args.workload]
+    sample_nnz = min(w.nnz, max(20_000, int(4.0e8 / w.k)))
+    frac = sample_nnz / w.nnz
+    m = max(8, int(math.ceil(w.m * min(1.0, frac * 4))))
+    n = max(8, int(math.ceil(w.n * min(1.0, frac * 4))))
+    sw = W.scaled(w, w.name + "-cpu-sample", m, n, min(sample_nnz, m * n // 2))
+    tpl = W.make_template(sw, "cpu")
+    r, c, v = tpl.rows.numpy(), tpl.cols.numpy(), tpl.vals.numpy()
+    P, Q = tpl.P0.numpy(), tpl.Q0.numpy()
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        st = oracle.grad_step(sw.m, sw.n, sw.k, r, c, v, P, Q, sw.eta, sw.lam, sw.xi, sw.clip, sw.norm_p, sw.norm_q)
+        dt = time.perf_counter() - t0
+        P, Q = st.P, st.Q
+        if it >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    val = tpl.nnz * len(times) / total
+    sample = "%dx%d k=%d nnz=%d template with the recipe of %s (oracle grad_step, double, single thread)" % (
+        sw.m, sw.n, sw.k, tpl.nnz, args.workload)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=15.0):
+    """Times the oracle on a prefix of the template's (row-sorted) COO entries with the full factor
+    matrices; sized from a short calibration run so that it takes about budget_s seconds."""
+    import numpy as np
+    import oracle
+    nnz = tpl_dev.nnz
+    P, Q = P0.cpu().numpy(), Q0.cpu().numpy()
+
+    def run(count):
+        r = tpl_dev.rows[:count].cpu().numpy(); c = tpl_dev.cols[:count].cpu().numpy()
+        v = tpl_dev.vals[:count].cpu().numpy()
+        m_used = int(r.max()) + 1 if count else 1     # the prefix touches rows [0, m_used)
+        t0 = time.perf_counter()
+        oracle.grad_step(m_used, w.n, w.k, r, c, v, P[:m_used], Q, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
+        return time.perf_counter() - t0, m_used
+
+    count = min(nnz, 1_000_000)
+    t, m_used = run(count)
+    if t < 0.5 * budget_s and count < nnz:   # the first run also pays fixed costs: rescale once
+        count = int(min(nnz, count * budget_s / max(t, 1e-3)))
+        t, m_used = run(count)
+    return {"value": count / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d of %d row-sorted entries (rows 0..%d, all %d columns), one oracle grad_step, "
+                      "%.1f s" % (count, nnz, m_used - 1, w.n, t)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=os.environ.get("TSID_BENCH_WORKLOAD", "C5"))
+    ap.add_argument("--impl", default="tsid")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2608_00977_b200 import workloads as W
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, W)
+        return
+
+    import __graft_entry__ as G
+    from paper_2608_00977_b200 import binding as B
+    if rank == 0:
+        G.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    B.lib()
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+
+    w = W.CONFIGS[args.workload]
+    t0 = time.perf_counter()
+    tpl = W.make_template(w, dev, order="sorted")
+    torch.cuda.synchronize(dev)
+    t1 = time.perf_counter()
+    nnz = tpl.nnz
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    torch.cuda.synchronize(dev)
+    if rank == 0:
+        sys.stderr.write("[bench] %s: generated %d entries in %.1f s, layout pass %.2f s, workspace %.2f GB\n" % (
+            w.name, nnz, t1 - t0, time.perf_counter() - t1, T.workspace.numel() / 1e9))
+    path, launches = T.tsid_get_info()
+    P, Q = tpl.P0.clone(), tpl.Q0.clone()
+    stream = torch.cuda.current_stream(dev)
+
+    resident = nnz * 16 + (w.m + w.n) * w.k * 4
+    flush = resident < 4 * L2_BYTES
+    scrub = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        T.tsid_grad_step(P, Q)
+    T.tsid_check()
+    T.tsid_set_profiling(True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    ms = 0.0
+    if flush:
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in evs:
+            scrub.fill_(1)
+            a.record(stream)
+            T.tsid_grad_step(P, Q)
+            b.record(stream)
+        barrier()
+        ms = sum(a.elapsed_time(b) for a, b in evs)
+    else:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.steps):
+            T.tsid_grad_step(P, Q)
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b)
+    clocks = sampler.stop()
+    nrec, row_ms, col_ms, upd_ms = T.tsid_get_pass_times()
+    T.tsid_set_profiling(False)
+    T.tsid_check()
+
+    if dist is not None:
+        tms = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+    value = world * nnz * args.steps / (ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (the gather-reduce pass: two launches per step) ----------
+    peak, peak_kind = load_peaks()
+    nseg_row = w.m + nnz // 1024
+    nseg_col = w.n + nnz // 1024
+    b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col)
+    pass_ms = (row_ms + col_ms) / max(1, 2 * nrec)
+    bytes_per_launch = (b_row + b_col) / 2
+    achieved = bytes_per_launch / (pass_ms * 1e-3) / 1e9 if pass_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "pass_kernel (CSR row pass + CSC column pass, 2 launches per step)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_source": "of %s" % peak_kind, "traffic": NCU_TRAFFIC_PER_LAUNCH.get(args.workload),
+                "alg_bytes_per_launch": bytes_per_launch, "avg_launch_ms": pass_ms,
+                "row_pass": {"ms": row_ms / max(1, nrec), "alg_bytes": b_row,
+                             "gbs": b_row / (row_ms / max(1, nrec) * 1e-3) / 1e9 if row_ms else None},
+                "col_pass": {"ms": col_ms / max(1, nrec), "alg_bytes": b_col,
+                             "gbs": b_col / (col_ms / max(1, nrec) * 1e-3) / 1e9 if col_ms else None},
+                "update": {"ms": upd_ms / max(1, nrec), "alg_bytes": b_upd,
+                           "gbs": b_upd / (upd_ms / max(1, nrec) * 1e-3) / 1e9 if upd_ms else None},
+                "step_alg_bytes": b_row + b_col + b_upd,
+                "step_frac": (b_row + b_col + b_upd) / (ms / args.steps * 1e-3) / 1e9 / peak,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # ---- end to end: host buffers through tsid_fit_host ----------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        epochs = args.e2e_epochs or w.epochs
+        cfg = B.make_config(w.m, w.n, w.k, nnz, prec, B.TSID_PATH_SPARSE, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
+        T.tsid_destroy()
+        del T
+        torch.cuda.empty_cache()
+        hb = [x.cpu().pin_memory() for x in (tpl.rows, tpl.cols, tpl.vals)]
+        hP0, hQ0 = tpl.P0.cpu(), tpl.Q0.cpu()
+        hP, hQ = hP0.clone().pin_memory(), hQ0.clone().pin_memory()
+        ws = torch.empty(B.tsid_workspace_bytes_host(cfg) + 256, dtype=torch.uint8, device=dev)
+        reps = 2
+        barrier()
+        t_e2e = 0.0
+        for rep in range(reps + 1):
+            hP.copy_(hP0); hQ.copy_(hQ0)
+            torch.cuda.synchronize(dev)
+            t0 = time.perf_counter()
+            B.tsid_fit_host(cfg, hb[0], hb[1], hb[2], hP, hQ, epochs, ws)
+            torch.cuda.synchronize(dev)
+            if rep > 0:   # the first call warms the pinned pages and the allocator
+                t_e2e += time.perf_counter() - t0
+        if dist is not None:
+            tt = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            t_e2e = float(tt.item())
+        h2d = nnz * 12 + (w.m + w.n) * w.k * 4
+        d2h = (w.m + w.n) * w.k * 4
+        e2e = {"value": world * nnz * epochs * reps / t_e2e, "unit": UNIT,
+               "h2d_bytes_per_step": h2d / epochs, "d2h_bytes_per_step": d2h / epochs,
+               "epochs_per_call": epochs, "h2d_bytes_per_call": h2d, "d2h_bytes_per_call": d2h,
+               "s_per_call": t_e2e / reps,
+               "what": "tsid_fit_host: pinned host COO + factors -> device, layout pass, epochs steps, factors -> host"}
+        del ws
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(w, tpl, tpl.P0, tpl.Q0)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision == "bf16" else "f32",
+                "data": "synthetic",
+                "config": {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": nnz,
+                           "precision": "bf16 shadow factors, fp32 master and accumulation" if w.precision == "bf16" else "fp32",
+                           "path": "sparse" if path == B.TSID_PATH_SPARSE else "dense_tc",
+                           "step": "tsid_grad_step (eta=%g lambda=%g xi=%g clip=%d norm=%d/%d)" % (
+                               w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q),
+                           "l2": "L2 flushed between timed steps (resident set %.0f MB)" % (resident / 1e6) if flush
+                                 else "inputs larger than L2 (resident set %.1f GB), steps timed back to back" % (resident / 1e9),
+                           "replicas": world},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches * args.steps,
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -140,6 +140,20 @@ tsid_status_t tsid_loss(tsid_template_t *t, const float *d_P, const float *d_Q, 
  * (TSID_ERR_NONFINITE, TSID_ERR_CUDA) or TSID_OK. */
 tsid_status_t tsid_check(tsid_template_t *t);
 
+/* The whole of Stage I from HOST arrays in one call (Sec. 5.1, "Stage I Execution Example":
+ * move the COO triples to the device, initialise from the given P, Q, iterate, return the
+ * factors).  h_rows/h_cols/h_vals (nnz each) and h_P (m x k), h_Q (n x k) are HOST pointers
+ * (pinned memory makes the copies asynchronous); h_P, h_Q are overwritten with the fitted
+ * factors.  cfg.workspace must hold tsid_workspace_bytes_host(cfg) bytes of DEVICE memory:
+ * the template's workspace followed by the staged triples and factors.  Copies in, builds the
+ * layout, runs `epochs` steps, optionally evaluates the SSE (host double), copies the factors
+ * back and synchronises.  Errors as in tsid_template_create / tsid_fit; message via
+ * tsid_last_error(NULL). */
+tsid_status_t tsid_workspace_bytes_host(const tsid_config_t *cfg, size_t *h_bytes_out);
+tsid_status_t tsid_fit_host(const tsid_config_t *cfg, const int32_t *h_rows, const int32_t *h_cols,
+                            const float *h_vals, float *h_P, float *h_Q, int32_t epochs,
+                            double *h_sse_or_null);
+
 /* Releases the host handle.  The workspace belongs to the caller.  NULL is accepted. */
 tsid_status_t tsid_destroy(tsid_template_t *t);
 
@@ -160,6 +174,15 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
 /* Which path the handle runs (tsid_path_t, never AUTO) and how many kernels one
  * tsid_grad_step launches. */
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
+
+/* Per-kernel timing for benchmarks.  tsid_set_profiling(t, 1) makes every following step record
+ * CUDA events on the template's stream right before and after its row pass, its column pass
+ * and its update kernel (at most 256 steps are kept); 0 turns it off and frees the events.
+ * tsid_get_pass_times synchronises, returns the number of recorded steps and the summed
+ * milliseconds of each of the three kernels over them, and restarts the recording. */
+tsid_status_t tsid_set_profiling(tsid_template_t *t, int32_t enable);
+tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms,
+                                  float *h_col_ms, float *h_update_ms);
 
 /* Message of the last failing call on this handle (or of the last failing create when
  * t == NULL).  Never NULL; valid until the next call on the same handle / thread. */

@@ -29,7 +29,8 @@ TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
 # every symbol include/tsid.h declares
 EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",
            "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
-           "tsid_last_error"]
+           "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
+           "tsid_get_pass_times"]
 
 
 class TsidConfig(C.Structure):
@@ -71,6 +72,10 @@ def lib():
         L.tsid_residuals.argtypes = [vp, vp, vp, vp]
         L.tsid_get_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.tsid_last_error.argtypes = [vp]
+        L.tsid_workspace_bytes_host.argtypes = [C.POINTER(TsidConfig), C.POINTER(C.c_size_t)]
+        L.tsid_fit_host.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, vp, C.c_int32, C.POINTER(C.c_double)]
+        L.tsid_set_profiling.argtypes = [vp, C.c_int32]
+        L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
         L.tsid_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name != "tsid_last_error":
@@ -185,6 +190,20 @@ class Template:
         lib().tsid_get_info(self.h, C.byref(p), C.byref(l))
         return p.value, l.value
 
+    def tsid_set_profiling(self, enable):
+        st = lib().tsid_set_profiling(self.h, int(enable))
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_get_pass_times(self):
+        """(steps, row_ms, col_ms, update_ms) summed over the recorded steps."""
+        n = C.c_int32(0)
+        a, b, c = C.c_float(0), C.c_float(0), C.c_float(0)
+        st = lib().tsid_get_pass_times(self.h, C.byref(n), C.byref(a), C.byref(b), C.byref(c))
+        if st != TSID_OK:
+            self._raise(st)
+        return n.value, a.value, b.value, c.value
+
     def tsid_get_layout(self):
         """Copies of the layout arrays as torch tensors (row_ptr, col_idx, val_csr, col_ptr, row_idx,
         val_csc, perm)."""
@@ -214,6 +233,41 @@ class Template:
             self.tsid_destroy()
         except Exception:
             pass
+
+
+def tsid_workspace_bytes_host(cfg: TsidConfig) -> int:
+    out = C.c_size_t(0)
+    st = lib().tsid_workspace_bytes_host(C.byref(cfg), C.byref(out))
+    if st != TSID_OK:
+        raise TsidError(st, lib().tsid_last_error(None).decode())
+    return out.value
+
+
+def tsid_fit_host(cfg: TsidConfig, rows, cols, vals, P, Q, epochs, workspace: torch.Tensor,
+                  stream=None, want_sse=False):
+    """Host-buffer call: rows/cols/vals/P/Q are CPU tensors (pinned for asynchronous copies); P, Q are
+    overwritten with the fitted factors.  `workspace` is a CUDA uint8 tensor of at least
+    tsid_workspace_bytes_host(cfg) + 256 bytes.  Returns the SSE if requested."""
+    for t, dt, nm in ((rows, torch.int32, "rows"), (cols, torch.int32, "cols"), (vals, torch.float32, "vals"),
+                      (P, torch.float32, "P"), (Q, torch.float32, "Q")):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous CPU tensor of %s" % (nm, dt))
+    need = tsid_workspace_bytes_host(cfg)
+    base = (workspace.data_ptr() + 255) & ~255
+    if workspace.numel() - (base - workspace.data_ptr()) < need:
+        raise ValueError("workspace too small: need %d bytes" % need)
+    c = TsidConfig.from_buffer_copy(cfg)
+    stream = stream if stream is not None else torch.cuda.current_stream(workspace.device)
+    c.stream = stream.cuda_stream
+    c.workspace = base
+    c.workspace_bytes = need
+    sse = C.c_double(0)
+    with torch.cuda.device(workspace.device):
+        st = lib().tsid_fit_host(C.byref(c), rows.data_ptr(), cols.data_ptr(), vals.data_ptr(), P.data_ptr(),
+                                 Q.data_ptr(), int(epochs), C.byref(sse) if want_sse else None)
+    if st != TSID_OK:
+        raise TsidError(st, lib().tsid_last_error(None).decode())
+    return sse.value if want_sse else None
 
 
 def template_from_workload(tpl, path=TSID_PATH_AUTO, flags=0, precision=None) -> Template:

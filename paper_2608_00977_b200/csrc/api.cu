@@ -222,9 +222,123 @@ tsid_status_t tsid_check(tsid_template_t *t) {
   return TSID_OK;
 }
 
+static void prof_release(tsid_template *t) {
+  if (t->prof.ev) {
+    for (int i = 0; i < kProfSteps * EV_PER_STEP; ++i) cudaEventDestroy(t->prof.ev[i]);
+    delete[] t->prof.ev;
+    t->prof.ev = nullptr;
+  }
+  t->prof.on = false;
+  t->prof.nsteps = 0;
+}
+
 tsid_status_t tsid_destroy(tsid_template_t *t) {
+  if (t) prof_release(t);
   delete t;
   return TSID_OK;
+}
+
+tsid_status_t tsid_set_profiling(tsid_template_t *t, int32_t enable) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (!enable) { prof_release(t); return TSID_OK; }
+  if (!t->prof.ev) {
+    t->prof.ev = new (std::nothrow) cudaEvent_t[kProfSteps * EV_PER_STEP];
+    if (!t->prof.ev) return fail(t, TSID_ERR_OOM, "host allocation failed");
+    for (int i = 0; i < kProfSteps * EV_PER_STEP; ++i) {
+      cudaError_t e = cudaEventCreate(&t->prof.ev[i]);
+      if (e != cudaSuccess) return cuda_fail(t, e);
+    }
+  }
+  t->prof.on = true;
+  t->prof.nsteps = 0;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms, float *h_col_ms,
+                                  float *h_update_ms) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (!t->prof.on) return fail(t, TSID_ERR_INVALID_ARG, "profiling is off");
+  cudaError_t e = cudaStreamSynchronize(t->stream);
+  if (e != cudaSuccess) return cuda_fail(t, e);
+  double acc[3] = {0, 0, 0};
+  for (int sidx = 0; sidx < t->prof.nsteps; ++sidx) {
+    for (int q = 0; q < 3; ++q) {
+      float ms = 0.f;
+      e = cudaEventElapsedTime(&ms, t->prof.ev[sidx * EV_PER_STEP + 2 * q], t->prof.ev[sidx * EV_PER_STEP + 2 * q + 1]);
+      if (e != cudaSuccess) return cuda_fail(t, e);
+      acc[q] += ms;
+    }
+  }
+  if (h_steps) *h_steps = t->prof.nsteps;
+  if (h_row_ms) *h_row_ms = (float)acc[0];
+  if (h_col_ms) *h_col_ms = (float)acc[1];
+  if (h_update_ms) *h_update_ms = (float)acc[2];
+  t->prof.nsteps = 0;
+  return TSID_OK;
+}
+
+// Device memory the host-buffer call needs: the template's own workspace, then the staged COO
+// triples and the two factor matrices.
+static size_t host_extra_bytes(const tsid_config_t &c) {
+  Carver cv(nullptr);
+  const size_t nz = c.nnz ? (size_t)c.nnz : 1;
+  cv.take<int32_t>(nz); cv.take<int32_t>(nz); cv.take<float>(nz);
+  cv.take<float>((size_t)c.m * c.k); cv.take<float>((size_t)c.n * c.k);
+  return cv.off;
+}
+
+tsid_status_t tsid_workspace_bytes_host(const tsid_config_t *cfg, size_t *h_bytes_out) {
+  size_t base = 0;
+  tsid_status_t st = tsid_workspace_bytes(cfg, &base);
+  if (st != TSID_OK) return st;
+  *h_bytes_out = base + host_extra_bytes(*cfg);
+  return TSID_OK;
+}
+
+tsid_status_t tsid_fit_host(const tsid_config_t *cfg, const int32_t *h_rows, const int32_t *h_cols,
+                            const float *h_vals, float *h_P, float *h_Q, int32_t epochs, double *h_sse_or_null) {
+  size_t base = 0, total = 0;
+  tsid_status_t st = tsid_workspace_bytes(cfg, &base);
+  if (st != TSID_OK) return st;
+  tsid_workspace_bytes_host(cfg, &total);
+  if (!h_P || !h_Q || (cfg->nnz > 0 && (!h_rows || !h_cols || !h_vals)))
+    return fail(nullptr, TSID_ERR_INVALID_ARG, "host pointer is null");
+  if (epochs < 0) return fail(nullptr, TSID_ERR_INVALID_ARG, "epochs must be >= 0");
+  if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255u))
+    return fail(nullptr, TSID_ERR_INVALID_ARG, "workspace is null or not 256-byte aligned");
+  if (cfg->workspace_bytes < total) return fail(nullptr, TSID_ERR_OOM, "workspace smaller than tsid_workspace_bytes_host");
+  cudaStream_t s = static_cast<cudaStream_t>(cfg->stream);
+  Carver cv(static_cast<char *>(cfg->workspace) + base);
+  const size_t nnz = (size_t)cfg->nnz, nz = nnz ? nnz : 1;
+  int32_t *d_rows = cv.take<int32_t>(nz), *d_cols = cv.take<int32_t>(nz);
+  float *d_vals = cv.take<float>(nz);
+  const size_t pb = (size_t)cfg->m * cfg->k * sizeof(float), qb = (size_t)cfg->n * cfg->k * sizeof(float);
+  float *d_P = cv.take<float>(pb / 4), *d_Q = cv.take<float>(qb / 4);
+  cudaError_t e = cudaSuccess;
+  if (nnz) {
+    e = cudaMemcpyAsync(d_rows, h_rows, nnz * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_cols, h_cols, nnz * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_vals, h_vals, nnz * 4, cudaMemcpyHostToDevice, s);
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_P, h_P, pb, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_Q, h_Q, qb, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e);
+  tsid_config_t c2 = *cfg;
+  c2.workspace_bytes = base;
+  tsid_template *t = nullptr;
+  st = tsid_template_create(&c2, d_rows, d_cols, d_vals, &t);
+  if (st != TSID_OK) return st;
+  st = tsid_fit(t, d_P, d_Q, epochs, 0, nullptr);
+  if (st == TSID_OK && h_sse_or_null) st = tsid_loss(t, d_P, d_Q, h_sse_or_null, nullptr);
+  if (st == TSID_OK) {
+    e = cudaMemcpyAsync(h_P, d_P, pb, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_Q, d_Q, qb, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) st = tsid_check(t);
+    if (e != cudaSuccess) st = cuda_fail(nullptr, e);
+  }
+  if (st != TSID_OK) snprintf(g_create_err, 256, "%s", t->err);
+  tsid_destroy(t);
+  return st;
 }
 
 tsid_status_t tsid_get_layout(tsid_template_t *t, const int64_t **d_row_ptr, const int32_t **d_col_idx,

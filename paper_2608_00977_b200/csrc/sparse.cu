@@ -362,6 +362,11 @@ cudaError_t launch_pass(tsid_template *t, const Side &sd, const void *stage, con
   return launch_pass_k<false, MODE>(t->stream, sd, stage, gather, k, G, t->partial, e_out, red);
 }
 
+inline void prof_mark(tsid_template *t, int which) {
+  if (t->prof.on && t->prof.nsteps < kProfSteps)
+    cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + which], t->stream);
+}
+
 inline int ew_grid(int64_t n) {
   int64_t g = (n + 255) / 256;
   if (g < 1) g = 1;
@@ -383,11 +388,15 @@ cudaError_t sparse_grad(tsid_template *t, const float *d_P, const float *d_Q, fl
   const bool bf = t->cfg.precision == TSID_BF16_SHADOW;
   const void *Ps = bf ? (const void *)t->rowside.shadow : (const void *)d_P;
   const void *Qs = bf ? (const void *)t->colside.shadow : (const void *)d_Q;
+  prof_mark(t, EV_ROW0);
   CK(launch_pass<MODE_GRAD>(t, t->rowside, Ps, Qs, GP, nullptr, nullptr));
+  prof_mark(t, EV_ROW1);
   if (t->rowside.nsplit > 0)
     fixup_kernel<<<t->rowside.nsplit, 128, 0, t->stream>>>(t->rowside.splits, t->rowside.nsplit, t->partial, GP,
                                                            t->cfg.k);
+  prof_mark(t, EV_COL0);
   CK(launch_pass<MODE_GRAD>(t, t->colside, Qs, Ps, GQ, nullptr, nullptr));
+  prof_mark(t, EV_COL1);
   if (t->colside.nsplit > 0)
     fixup_kernel<<<t->colside.nsplit, 128, 0, t->stream>>>(t->colside.splits, t->colside.nsplit, t->partial, GQ,
                                                            t->cfg.k);
@@ -398,8 +407,11 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
   const tsid_config_t &c = t->cfg;
   UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4};
   UpdSide b{d_Q, GQ, t->colside.scale, t->colside.shadow, (int64_t)c.n * c.k / 4};
+  prof_mark(t, EV_UPD0);
   update_kernel<<<ew_grid(a.n4 + b.n4), 256, 0, t->stream>>>(a, b, c.k / 4, c.eta, 2.0f * c.lambda, c.xi, c.clip,
                                                              t->flags);
+  prof_mark(t, EV_UPD1);
+  if (t->prof.on && t->prof.nsteps < kProfSteps) t->prof.nsteps++;
   return cudaGetLastError();
 }
 

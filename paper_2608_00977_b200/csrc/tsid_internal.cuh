@@ -50,6 +50,16 @@ struct Side {
 
 struct DenseState;  // dense_tc.cu
 
+// Optional per-kernel timing: CUDA events recorded on the template's stream right around the
+// row pass, the column pass and the update kernel of each step (up to kProfSteps steps).
+constexpr int kProfSteps = 256;
+enum { EV_ROW0 = 0, EV_ROW1, EV_COL0, EV_COL1, EV_UPD0, EV_UPD1, EV_PER_STEP };
+struct Prof {
+  bool on = false;
+  int nsteps = 0;
+  cudaEvent_t *ev = nullptr;  // [kProfSteps * EV_PER_STEP], host-side handles
+};
+
 }  // namespace tsid
 
 struct tsid_template {
@@ -67,6 +77,7 @@ struct tsid_template {
   int32_t red_cap;
   int32_t *flags;     // device flags: [0] range, [1] unsorted, [2] duplicate, [3] non-finite
   tsid::DenseState *dense;
+  tsid::Prof prof;
   char err[256];
 };
 
