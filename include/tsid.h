@@ -56,8 +56,10 @@ typedef enum {
   TSID_ERR_OOM = 5,          /* workspace smaller than tsid_workspace_bytes               */
   TSID_ERR_CUDA = 6,         /* a CUDA runtime call failed (message in tsid_last_error)   */
   TSID_ERR_UNSUPPORTED = 7,  /* configuration outside the limits above                    */
-  TSID_ERR_NONFINITE = 8     /* an updated factor became inf/nan (reported by tsid_check, */
+  TSID_ERR_NONFINITE = 8,    /* an updated factor became inf/nan (reported by tsid_check, */
                              /* tsid_loss and tsid_fit with loss_every > 0)               */
+  TSID_ERR_TOO_LARGE = 9     /* tsid_sse_noalloc: more entries than its built-in scratch   */
+                             /* covers (the call did nothing)                             */
 } tsid_status_t;
 
 /* Storage precision of the factor values the two gradient passes READ.  The
@@ -183,6 +185,34 @@ tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *
 tsid_status_t tsid_set_profiling(tsid_template_t *t, int32_t enable);
 tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms,
                                   float *h_col_ms, float *h_update_ms);
+
+/* (The paper has no counterpart for this call; it exists for callers that cannot allocate.)
+ * SSE = sum_Omega (r_ij - p_i . q_j)^2 of a template given as raw COO triples, with fp32 factors,
+ * WITHOUT a handle, a workspace or any allocation.  It is meant for code that is handed device
+ * pointers and a stream but may not create device memory: a monitoring hook inside a process
+ * whose framework owns the whole GPU through its own pool, a latency-critical loop that cannot
+ * afford the device-wide synchronisation an allocate/free pair brings, a plug-in with no
+ * allocator access.  The partial sums the reduction needs live in a fixed 512 KiB array that is
+ * part of the library image on every GPU that loads it (until the process exits).
+ *   - All d_* pointers are device memory of the CURRENT device: d_rows, d_cols (int32[nnz],
+ *     indices must be in range: they are not checked), d_vals (fp32[nnz]), d_P (m x k), d_Q
+ *     (n x k) fp32 row-major and 16-byte aligned, k a multiple of 4 in [4, 256].  The result is
+ *     written to d_sse_out (one double, device memory, 8-byte aligned) by work enqueued on
+ *     `stream`; the call does not synchronise.  Residuals are fp32, squares are added in double
+ *     in a fixed order (deterministic).
+ *   - Limit: nnz <= 67,108,864 (65,536 partial sums of 1,024 entries).  Larger templates are
+ *     refused with TSID_ERR_TOO_LARGE before anything is launched; use tsid_loss for those.
+ *   - The first call on each device looks up the device address of the built-in array (a
+ *     runtime query, no allocation).  Make that first call at start-up, with the device current,
+ *     before any stream capture is begun on the thread.
+ *   - Every call on a device uses the same array.  Calls whose GPU work can overlap (two
+ *     streams, two host threads) race on it: serialise them.  The array keeps the previous
+ *     call's contents, which is harmless: each call overwrites every slot it reads.
+ *   - Other statuses: TSID_ERR_INVALID_ARG (null or misaligned pointer, bad size),
+ *     TSID_ERR_UNSUPPORTED (k outside the limits, device ordinal above 63), TSID_ERR_CUDA. */
+tsid_status_t tsid_sse_noalloc(int32_t m, int32_t n, int32_t k, int64_t nnz, const int32_t *d_rows,
+                               const int32_t *d_cols, const float *d_vals, const float *d_P,
+                               const float *d_Q, void *stream, double *d_sse_out);
 
 /* Message of the last failing call on this handle (or of the last failing create when
  * t == NULL).  Never NULL; valid until the next call on the same handle / thread. */

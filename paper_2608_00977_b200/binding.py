@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libtsid.so")
 TSID_OK = 0
 STATUS_NAMES = ["TSID_OK", "TSID_ERR_INVALID_ARG", "TSID_ERR_INDEX_RANGE", "TSID_ERR_DUPLICATE",
                 "TSID_ERR_UNSORTED", "TSID_ERR_OOM", "TSID_ERR_CUDA", "TSID_ERR_UNSUPPORTED",
-                "TSID_ERR_NONFINITE"]
+                "TSID_ERR_NONFINITE", "TSID_ERR_TOO_LARGE"]
+TSID_ERR_TOO_LARGE = 9
 (TSID_ERR_INVALID_ARG, TSID_ERR_INDEX_RANGE, TSID_ERR_DUPLICATE, TSID_ERR_UNSORTED, TSID_ERR_OOM,
  TSID_ERR_CUDA, TSID_ERR_UNSUPPORTED, TSID_ERR_NONFINITE) = range(1, 9)
 TSID_F32, TSID_BF16_SHADOW = 0, 1
@@ -30,7 +31,7 @@ TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
 EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",
            "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
-           "tsid_get_pass_times"]
+           "tsid_get_pass_times", "tsid_sse_noalloc"]
 
 
 class TsidConfig(C.Structure):
@@ -76,6 +77,7 @@ def lib():
         L.tsid_fit_host.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, vp, C.c_int32, C.POINTER(C.c_double)]
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
         L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
+        L.tsid_sse_noalloc.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
         L.tsid_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name != "tsid_last_error":
@@ -268,6 +270,25 @@ def tsid_fit_host(cfg: TsidConfig, rows, cols, vals, P, Q, epochs, workspace: to
     if st != TSID_OK:
         raise TsidError(st, lib().tsid_last_error(None).decode())
     return sse.value if want_sse else None
+
+
+def tsid_sse_noalloc(m, n, k, rows, cols, vals, P, Q, out, stream=None):
+    """SSE of a COO template without a handle or workspace: `out` (CUDA float64 tensor with one element)
+    receives the result asynchronously on `stream`.  For callers that may not allocate device memory: this
+    wrapper allocates nothing either (all tensors, the output included, come from the caller)."""
+    nnz = int(rows.numel())
+    _check_tensor(rows, torch.int32, nnz, "rows")
+    _check_tensor(cols, torch.int32, nnz, "cols")
+    _check_tensor(vals, torch.float32, nnz, "vals")
+    _check_tensor(P, torch.float32, m * k, "P")
+    _check_tensor(Q, torch.float32, n * k, "Q")
+    _check_tensor(out, torch.float64, 1, "out")
+    stream = stream if stream is not None else torch.cuda.current_stream(P.device)
+    with torch.cuda.device(P.device):
+        st = lib().tsid_sse_noalloc(m, n, k, nnz, rows.data_ptr(), cols.data_ptr(), vals.data_ptr(), P.data_ptr(),
+                                    Q.data_ptr(), stream.cuda_stream, out.data_ptr())
+    if st != TSID_OK:
+        raise TsidError(st, "tsid_sse_noalloc refused or failed")
 
 
 def template_from_workload(tpl, path=TSID_PATH_AUTO, flags=0, precision=None) -> Template:
