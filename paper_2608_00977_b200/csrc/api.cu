@@ -169,6 +169,7 @@ static tsid_status_t loss_sync(tsid_template *t, const float *d_P, const float *
   if (e != cudaSuccess) return cuda_fail(t, e);
   *sse = h[0];
   *sq = h[1];
+  if (hf[FLAG_TIMEOUT]) return fail(t, TSID_ERR_CUDA, "a bounded device-side wait expired ");
   if (hf[FLAG_NONFINITE] || !(h[0] == h[0]) || !(h[1] == h[1]))
     return fail(t, TSID_ERR_NONFINITE, "a factor became non-finite");
   return TSID_OK;
@@ -218,6 +219,7 @@ tsid_status_t tsid_check(tsid_template_t *t) {
   cudaError_t e = cudaMemcpyAsync(hf, t->flags, sizeof(hf), cudaMemcpyDeviceToHost, t->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(t->stream);
   if (e != cudaSuccess) return cuda_fail(t, e);
+  if (hf[FLAG_TIMEOUT]) return fail(t, TSID_ERR_CUDA, "a bounded device-side wait expired ");
   if (hf[FLAG_NONFINITE]) return fail(t, TSID_ERR_NONFINITE, "a factor became non-finite");
   return TSID_OK;
 }

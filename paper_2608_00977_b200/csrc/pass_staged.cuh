@@ -1,0 +1,221 @@
+// Staged variant of the gradient pass.  Included by sparse.cu inside its namespace, after Geo,
+// Raw and the pass_kernel it mirrors.
+//
+// Same arithmetic and the same summation order as pass_kernel<MODE_GRAD> (bitwise identical
+// results), but the gathered factor rows travel global -> shared memory with 16-byte asynchronous
+// copies (cp.async, L2 only), NST chunks of ROWS rows deep.  The bytes in flight then live in
+// shared memory instead of registers; the k = 128 passes are bound by exactly that (gathers served
+// by L2 / HBM at several hundred ns each, 256 B per entry).  A CTA is ONE warp: segments differ in
+// length, and a multi-warp CTA keeps the shared memory of its finished warps idle until its longest
+// segment ends.  There is no barrier and no spin-wait: completion is cp.async.wait_group.
+#pragma once
+
+template <bool BF16, int VE>
+struct SRaw;  // reads a Raw vector from a shared-memory address
+template <>
+struct SRaw<false, 4> {
+  static __device__ __forceinline__ void load(Raw<false, 4> &r, uint32_t a) {
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.v.x), "=f"(r.v.y), "=f"(r.v.z), "=f"(r.v.w) : "r"(a));
+  }
+};
+template <>
+struct SRaw<true, 8> {
+  static __device__ __forceinline__ void load(Raw<true, 8> &r, uint32_t a) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.v.x), "=r"(r.v.y), "=r"(r.v.z), "=r"(r.v.w) : "r"(a));
+  }
+};
+template <>
+struct SRaw<true, 4> {
+  static __device__ __forceinline__ void load(Raw<true, 4> &r, uint32_t a) {
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(r.v.x), "=r"(r.v.y) : "r"(a));
+  }
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int KP, bool BF16, int NST, int ROWS>
+__global__ void __launch_bounds__(32)
+pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__restrict__ idx,
+                   const float *__restrict__ val, const void *__restrict__ stage_v,
+                   const void *__restrict__ gather_v, int k, float *__restrict__ G,
+                   float *__restrict__ partial) {
+  using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+  constexpr int GROUP = Geo<KP>::GROUP, EPL = Geo<KP>::EPL, EPW = Geo<KP>::EPW;
+  constexpr int VE = BF16 ? (EPL >= 8 ? 8 : 4) : 4;
+  constexpr int NV = EPL / VE;
+  constexpr int SLOT = KP * (int)sizeof(T);  // bytes reserved per gathered row
+  constexpr int STAGE = ROWS * SLOT;         // one chunk
+  constexpr int PIECES = SLOT / 16;          // 16-byte pieces per row
+  constexpr int NCP = ROWS * PIECES / 32;    // cp.async instructions per lane per chunk
+  static_assert(ROWS % EPW == 0 && (ROWS / EPW) % 2 == 0, "chunk must hold an even number of warp iterations");
+  static_assert(PIECES <= 32 && 32 % PIECES == 0 && ROWS * PIECES % 32 == 0, "piece mapping");
+  using R = Raw<BF16, VE>;
+  const T *stage = static_cast<const T *>(stage_v);
+  const T *gat = static_cast<const T *>(gather_v);
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int lane = threadIdx.x;
+  const uint32_t sbase = smem_u32(smem_raw);
+  const int warp = blockIdx.x;
+  if (warp >= nseg) return;
+
+  const int g = lane / GROUP, s = lane % GROUP;
+  const Segment sg = segs[warp];
+  const int pr = lane / PIECES, pp = lane % PIECES;  // this lane's (row within a copy instruction, piece)
+  const bool pvalid = pp * 16 < k * (int)sizeof(T);
+
+  bool cv[NV];
+  int co[NV];
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    co[c] = c * GROUP * VE + s * VE;
+    cv[c] = co[c] < k;
+  }
+  float x[EPL], acc[EPL];
+  {
+    const T *xr = stage + (size_t)sg.row * k;
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+      R r;
+      r.zero();
+      if (cv[c]) r.load(xr + co[c]);
+      r.unpack(x + c * VE);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) acc[i] = 0.f;
+
+  const int32_t *ip = idx + sg.begin;
+  const float *vp = val + sg.begin;
+  const int len = sg.len;
+  const int nchunks = (len + ROWS - 1) / ROWS;
+
+  float vring[NST];
+#pragma unroll
+  for (int u = 0; u < NST; ++u) vring[u] = 0.f;
+
+  // Copies of chunk c (lane l < ROWS holds the index of its l-th entry in j) into stage st.
+  // Always commits a group, also for chunks past the end, so that wait_group counts stay aligned.
+  auto issue = [&](int c, int st, int32_t j) {
+    if (c < nchunks) {
+      const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
+      const uint32_t dst0 = sbase + st * STAGE + pp * 16;
+#pragma unroll
+      for (int q = 0; q < NCP; ++q) {
+        const int r = q * (32 / PIECES) + pr;
+        const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
+        if (r < nv && pvalid)
+          cp_async16(dst0 + r * SLOT, reinterpret_cast<const unsigned char *>(gat + (size_t)jr * k) + pp * 16);
+      }
+    }
+    cp_async_commit();
+  };
+  auto load_iv = [&](int c, int32_t &j, float &r) {
+    j = 0;
+    r = 0.f;
+    if (lane < ROWS && c * ROWS + lane < len) { j = __ldcs(ip + c * ROWS + lane); r = __ldcs(vp + c * ROWS + lane); }
+  };
+
+  // prologue: chunks 0 .. NST-2 in flight, indices of chunk NST-1 loaded
+  int32_t nj;
+  float nr;
+#pragma unroll
+  for (int u = 0; u < NST - 1; ++u) {
+    int32_t j;
+    load_iv(u, j, vring[u]);
+    issue(u, u, j);
+  }
+  load_iv(NST - 1, nj, nr);
+
+  for (int c0 = 0; c0 < nchunks; c0 += NST) {
+#pragma unroll
+    for (int u = 0; u < NST; ++u) {
+      const int c = c0 + u;
+      if (c < nchunks) {
+        // keep the pipe full: chunk c+NST-1 goes into the stage that chunk c-1 released
+        const int cn = c + NST - 1;
+        const int sn = (u + NST - 1) % NST;
+        vring[sn] = nr;
+        issue(cn, sn, nj);
+        load_iv(cn + 1, nj, nr);
+        cp_async_wait<NST - 1>();  // all but the newest NST-1 groups are done: chunk c has landed
+        __syncwarp();
+
+        const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
+        const float myr = vring[u];
+        const uint32_t sst = sbase + u * STAGE;
+        const int iters = (nv + EPW - 1) / EPW;
+        for (int it = 0; it < iters; it += 2) {
+          const int sa = it * EPW + g, sb = sa + EPW;
+          const float ra = __shfl_sync(0xffffffffu, myr, sa & 31);
+          const float rb = __shfl_sync(0xffffffffu, myr, sb & 31);
+          const bool va = sa < nv, vb = sb < nv;
+          R ya[NV], yb[NV];
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            ya[q].zero();
+            yb[q].zero();
+            if (va && cv[q]) SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+            if (vb && cv[q]) SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+          }
+          float fa[EPL], fb[EPL];
+#pragma unroll
+          for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+          float da = 0.f, db = 0.f;
+#pragma unroll
+          for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+#pragma unroll
+          for (int o = GROUP / 2; o > 0; o >>= 1) {
+            da += __shfl_xor_sync(0xffffffffu, da, o);
+            db += __shfl_xor_sync(0xffffffffu, db, o);
+          }
+          const float ea = va ? ra - da : 0.f;
+          const float eb = vb ? rb - db : 0.f;
+#pragma unroll
+          for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
+#pragma unroll
+          for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
+        }
+        __syncwarp();  // every lane is done reading this stage before it is refilled
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+#pragma unroll
+  for (int o = GROUP; o < 32; o <<= 1) {
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+  }
+  if (g == 0) {
+    float *dst = sg.slot < 0 ? G + (size_t)sg.row * k : partial + (size_t)sg.slot * k;
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+      if (cv[c]) {
+#pragma unroll
+        for (int q = 0; q < VE / 4; ++q)
+          *reinterpret_cast<float4 *>(dst + co[c] + 4 * q) =
+              make_float4(acc[c * VE + 4 * q], acc[c * VE + 4 * q + 1], acc[c * VE + 4 * q + 2],
+                          acc[c * VE + 4 * q + 3]);
+      }
+    }
+  }
+}
+
+template <int KP, bool BF16, int NST, int ROWS>
+cudaError_t launch_staged_t(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+  using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+  constexpr int smem = NST * ROWS * KP * (int)sizeof(T);
+  auto kern = pass_staged_kernel<KP, BF16, NST, ROWS>;
+  CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  kern<<<sd.nseg, 32, smem, t->stream>>>(sd.segs, sd.nseg, sd.idx, sd.val, stage, gather, t->cfg.k, G, t->partial);
+  return cudaGetLastError();
+}

@@ -336,7 +336,7 @@ template <int KP, bool BF16, int MODE>
 cudaError_t launch_pass_t(cudaStream_t st, const Side &sd, const void *stage, const void *gather, int k,
                           float *G, float *partial, float *e_out, double *red) {
   if (sd.nseg <= 0) return cudaSuccess;
-  const int wpb = 8;
+  const int wpb = 2;  // small CTAs: segments differ in length, a CTA lives as long as its longest one
   const int grid = (sd.nseg + wpb - 1) / wpb;
   pass_kernel<KP, BF16, MODE><<<grid, wpb * 32, 0, st>>>(sd.segs, sd.nseg, sd.idx, sd.val, stage, gather, k, G,
                                                          partial, e_out, red);
@@ -353,9 +353,36 @@ cudaError_t launch_pass_k(cudaStream_t st, const Side &sd, const void *stage, co
   return launch_pass_t<256, BF16, MODE>(st, sd, stage, gather, k, G, partial, e_out, red);
 }
 
+#include "pass_staged.cuh"
+
+// Staged gradient pass for every (KP, precision) whose factor row fits the copy mapping (<= 512 B).
+// Chunk depth measured on B200: two stages; 16-row chunks for 256-byte rows and wider (more CTAs
+// per SM matter more than deeper chunks), 32-row chunks below.  Returns cudaErrorNotSupported when
+// there is no staged instantiation (fp32 with k > 128): the caller then uses the direct kernel.
+cudaError_t launch_staged(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+  if (sd.nseg <= 0) return cudaSuccess;
+  const int k = t->cfg.k;
+  if (t->cfg.precision == TSID_BF16_SHADOW) {
+    if (k <= 16) return launch_staged_t<16, true, 2, 32>(t, sd, stage, gather, G);
+    if (k <= 32) return launch_staged_t<32, true, 2, 32>(t, sd, stage, gather, G);
+    if (k <= 64) return launch_staged_t<64, true, 2, 32>(t, sd, stage, gather, G);
+    if (k <= 128) return launch_staged_t<128, true, 2, 16>(t, sd, stage, gather, G);
+    return launch_staged_t<256, true, 2, 16>(t, sd, stage, gather, G);
+  }
+  if (k <= 16) return launch_staged_t<16, false, 2, 32>(t, sd, stage, gather, G);
+  if (k <= 32) return launch_staged_t<32, false, 2, 32>(t, sd, stage, gather, G);
+  if (k <= 64) return launch_staged_t<64, false, 2, 16>(t, sd, stage, gather, G);
+  if (k <= 128) return launch_staged_t<128, false, 2, 16>(t, sd, stage, gather, G);
+  return cudaErrorNotSupported;
+}
+
 template <int MODE>
 cudaError_t launch_pass(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G,
                         float *e_out, double *red) {
+  if (MODE == MODE_GRAD) {
+    cudaError_t e = launch_staged(t, sd, stage, gather, G);
+    if (e != cudaErrorNotSupported) return e;
+  }
   const int k = t->cfg.k;
   if (t->cfg.precision == TSID_BF16_SHADOW)
     return launch_pass_k<true, MODE>(t->stream, sd, stage, gather, k, G, t->partial, e_out, red);

@@ -83,7 +83,7 @@ struct tsid_template {
 
 namespace tsid {
 
-enum { FLAG_RANGE = 0, FLAG_UNSORTED = 1, FLAG_DUP = 2, FLAG_NONFINITE = 3, FLAG_COUNT = 8 };
+enum { FLAG_RANGE = 0, FLAG_UNSORTED = 1, FLAG_DUP = 2, FLAG_NONFINITE = 3, FLAG_TIMEOUT = 4, FLAG_COUNT = 8 };
 
 // Carves 256-byte aligned pieces out of the caller's workspace; with base == nullptr it
 // only measures.
