@@ -31,8 +31,11 @@ tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
   return TSID_OK;
 }
 
+// AUTO takes the dense tensor-core variant when the template qualifies for it and at least 5 % of
+// its cells are observed; the answer depends on cfg alone, so the workspace size is predictable.
 int resolve_path(const tsid_config_t &c) {
   if (c.path != TSID_PATH_AUTO) return c.path;
+  if (dense_qualifies(c) && (double)c.nnz >= 0.05 * (double)c.m * (double)c.n) return TSID_PATH_DENSE_TC;
   return TSID_PATH_SPARSE;
 }
 
@@ -67,6 +70,7 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
   t->partial = cv.take<float>((2 * per + 2) * k);
   t->red_cap = (int32_t)(2 + 2 * 256 + t->rowside.cap_seg);
   t->red = cv.take<double>(t->red_cap);
+  if (t->path == TSID_PATH_DENSE_TC) dense_carve(t, c, cv);
   // transient buffers of the layout pass
   ls.kA = cv.take<uint32_t>(nz); ls.kB = cv.take<uint32_t>(nz);
   ls.vA = cv.take<uint32_t>(nz); ls.vB = cv.take<uint32_t>(nz);
@@ -74,6 +78,10 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
   const size_t mx = (m > n ? m : n) + 2;
   ls.scanA = cv.take<uint32_t>(mx); ls.scanB = cv.take<uint32_t>(mx); ls.scanC = cv.take<uint32_t>(mx);
   ls.blocksums = cv.take<uint32_t>(kScanBlocksMax);
+}
+
+cudaError_t grad_any(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ) {
+  return t->path == TSID_PATH_DENSE_TC ? dense_grad(t, GP, GQ) : sparse_grad(t, d_P, d_Q, GP, GQ);
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -99,6 +107,11 @@ tsid_status_t tsid_workspace_bytes(const tsid_config_t *cfg, size_t *h_bytes_out
   if (st != TSID_OK) return st;
   tsid_template tmp;
   memset(static_cast<void *>(&tmp), 0, sizeof(tmp));
+  tmp.path = resolve_path(*cfg);
+  if (tmp.path == TSID_PATH_DENSE_TC && !dense_qualifies(*cfg)) {
+    snprintf(g_create_err, 256, "dense path needs bf16 shadows, k in {64, 128}, m and n multiples of 128");
+    return TSID_ERR_UNSUPPORTED;
+  }
   Carver cv(nullptr);
   LayoutScratch ls;
   carve_all(&tmp, *cfg, cv, ls);
@@ -119,7 +132,6 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
   tsid_workspace_bytes(cfg, &need);
   if (cfg->workspace_bytes < need) return fail(nullptr, TSID_ERR_OOM, "workspace smaller than tsid_workspace_bytes");
   const int path = resolve_path(*cfg);
-  if (path == TSID_PATH_DENSE_TC) return fail(nullptr, TSID_ERR_UNSUPPORTED, "dense tensor-core path not available for this template");
 
   tsid_template *t = new (std::nothrow) tsid_template;
   if (!t) return fail(nullptr, TSID_ERR_OOM, "host allocation failed");
@@ -127,6 +139,10 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
   t->cfg = *cfg;
   t->stream = static_cast<cudaStream_t>(cfg->stream);
   t->path = path;
+  if (path == TSID_PATH_DENSE_TC) {
+    t->dense = dense_new();
+    if (!t->dense) { delete t; return fail(nullptr, TSID_ERR_OOM, "host allocation failed"); }
+  }
   Carver cv(cfg->workspace);
   LayoutScratch ls;
   carve_all(t, *cfg, cv, ls);
@@ -139,7 +155,13 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
   if (hf[FLAG_DUP] && (cfg->flags & TSID_VALIDATE)) { delete t; return fail(nullptr, TSID_ERR_DUPLICATE, "duplicate (row, col) in Omega"); }
   e = build_segments(t, t->rowside, cfg->norm_p, ls);
   if (e == cudaSuccess) e = build_segments(t, t->colside, cfg->norm_q, ls);
-  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); delete t; return st; }
+  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+  if (path == TSID_PATH_DENSE_TC) {
+    int32_t bad = 0;
+    e = dense_build(t, &bad);
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+    if (bad) { tsid_destroy(t); return fail(nullptr, TSID_ERR_UNSUPPORTED, "a value is outside the fp16 range of the dense path"); }
+  }
   snprintf(t->err, 256, "ok");
   *out = t;
   return TSID_OK;
@@ -154,7 +176,7 @@ tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *
   float *GP = d_gradP_or_null ? d_gradP_or_null : t->rowside.G;
   float *GQ = d_gradQ_or_null ? d_gradQ_or_null : t->colside.G;
   cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
-  if (e == cudaSuccess) e = sparse_grad(t, d_P, d_Q, GP, GQ);
+  if (e == cudaSuccess) e = grad_any(t, d_P, d_Q, GP, GQ);
   if (e == cudaSuccess) e = sparse_update(t, d_P, d_Q, GP, GQ);
   return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
 }
@@ -191,7 +213,7 @@ tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epoch
   cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
   for (int ep = 0; ep < epochs && e == cudaSuccess; ++ep) {
     // the update kernel refreshes the shadows, so they stay current between epochs
-    e = sparse_grad(t, d_P, d_Q, t->rowside.G, t->colside.G);
+    e = grad_any(t, d_P, d_Q, t->rowside.G, t->colside.G);
     if (e == cudaSuccess) e = sparse_update(t, d_P, d_Q, t->rowside.G, t->colside.G);
     if (e == cudaSuccess && loss_every > 0 && (ep + 1) % loss_every == 0) {
       st = loss_sync(t, d_P, d_Q, &sse, &sq);
@@ -235,7 +257,7 @@ static void prof_release(tsid_template *t) {
 }
 
 tsid_status_t tsid_destroy(tsid_template_t *t) {
-  if (t) prof_release(t);
+  if (t) { prof_release(t); dense_delete(t->dense); }
   delete t;
   return TSID_OK;
 }
@@ -368,7 +390,7 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step) {
   if (!t) return TSID_ERR_INVALID_ARG;
   if (h_path) *h_path = t->path;
-  if (h_launches_per_step) *h_launches_per_step = sparse_launches_per_step(t);
+  if (h_launches_per_step) *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? 6 : sparse_launches_per_step(t);
   return TSID_OK;
 }
 

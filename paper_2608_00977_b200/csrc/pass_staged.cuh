@@ -108,12 +108,22 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
     if (c < nchunks) {
       const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
       const uint32_t dst0 = sbase + st * STAGE + pp * 16;
+      const unsigned char *src0 = reinterpret_cast<const unsigned char *>(gat) + pp * 16;
+      const size_t rowbytes = (size_t)k * sizeof(T);
+      if (k == KP && nv == ROWS) {
 #pragma unroll
-      for (int q = 0; q < NCP; ++q) {
-        const int r = q * (32 / PIECES) + pr;
-        const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
-        if (r < nv && pvalid)
-          cp_async16(dst0 + r * SLOT, reinterpret_cast<const unsigned char *>(gat + (size_t)jr * k) + pp * 16);
+        for (int q = 0; q < NCP; ++q) {
+          const int r = q * (32 / PIECES) + pr;
+          const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
+          cp_async16(dst0 + r * SLOT, src0 + (size_t)jr * rowbytes);
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < NCP; ++q) {
+          const int r = q * (32 / PIECES) + pr;
+          const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
+          if (r < nv && pvalid) cp_async16(dst0 + r * SLOT, src0 + (size_t)jr * rowbytes);
+        }
       }
     }
     cp_async_commit();
@@ -152,37 +162,69 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
         const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
         const float myr = vring[u];
         const uint32_t sst = sbase + u * STAGE;
-        const int iters = (nv + EPW - 1) / EPW;
-        for (int it = 0; it < iters; it += 2) {
-          const int sa = it * EPW + g, sb = sa + EPW;
-          const float ra = __shfl_sync(0xffffffffu, myr, sa & 31);
-          const float rb = __shfl_sync(0xffffffffu, myr, sb & 31);
-          const bool va = sa < nv, vb = sb < nv;
-          R ya[NV], yb[NV];
+        if (k == KP && nv == ROWS) {
+          // full chunk of full-width rows (the common case): no predicates, fully unrolled
 #pragma unroll
-          for (int q = 0; q < NV; ++q) {
-            ya[q].zero();
-            yb[q].zero();
-            if (va && cv[q]) SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
-            if (vb && cv[q]) SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+          for (int it = 0; it < ROWS / EPW; it += 2) {
+            const int sa = it * EPW + g, sb = sa + EPW;
+            const float ra = __shfl_sync(0xffffffffu, myr, sa);
+            const float rb = __shfl_sync(0xffffffffu, myr, sb);
+            R ya[NV], yb[NV];
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+              SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+              SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+            }
+            float fa[EPL], fb[EPL];
+#pragma unroll
+            for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+            float da = 0.f, db = 0.f;
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+#pragma unroll
+            for (int o = GROUP / 2; o > 0; o >>= 1) {
+              da += __shfl_xor_sync(0xffffffffu, da, o);
+              db += __shfl_xor_sync(0xffffffffu, db, o);
+            }
+            const float ea = ra - da, eb = rb - db;
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
           }
-          float fa[EPL], fb[EPL];
+        } else {
+          const int iters = (nv + EPW - 1) / EPW;
+          for (int it = 0; it < iters; it += 2) {
+            const int sa = it * EPW + g, sb = sa + EPW;
+            const float ra = __shfl_sync(0xffffffffu, myr, sa & 31);
+            const float rb = __shfl_sync(0xffffffffu, myr, sb & 31);
+            const bool va = sa < nv, vb = sb < nv;
+            R ya[NV], yb[NV];
 #pragma unroll
-          for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
-          float da = 0.f, db = 0.f;
+            for (int q = 0; q < NV; ++q) {
+              ya[q].zero();
+              yb[q].zero();
+              if (va && cv[q]) SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+              if (vb && cv[q]) SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+            }
+            float fa[EPL], fb[EPL];
 #pragma unroll
-          for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+            for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+            float da = 0.f, db = 0.f;
 #pragma unroll
-          for (int o = GROUP / 2; o > 0; o >>= 1) {
-            da += __shfl_xor_sync(0xffffffffu, da, o);
-            db += __shfl_xor_sync(0xffffffffu, db, o);
+            for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+#pragma unroll
+            for (int o = GROUP / 2; o > 0; o >>= 1) {
+              da += __shfl_xor_sync(0xffffffffu, da, o);
+              db += __shfl_xor_sync(0xffffffffu, db, o);
+            }
+            const float ea = va ? ra - da : 0.f;
+            const float eb = vb ? rb - db : 0.f;
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
           }
-          const float ea = va ? ra - da : 0.f;
-          const float eb = vb ? rb - db : 0.f;
-#pragma unroll
-          for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
-#pragma unroll
-          for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
         }
         __syncwarp();  // every lane is done reading this stage before it is refilled
       }

@@ -122,6 +122,14 @@ cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_
 cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
 int sparse_launches_per_step(const tsid_template *t);
 
+// dense tensor-core variant (dense_tc.cu)
+bool dense_qualifies(const tsid_config_t &c);
+DenseState *dense_new();
+void dense_delete(DenseState *d);
+void dense_carve(tsid_template *t, const tsid_config_t &c, Carver &cv);
+cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag);
+cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ);
+
 inline int bits_for(uint32_t maxval) {  // number of bits needed to represent values <= maxval
   int b = 0;
   while (b < 32 && (maxval >> b) != 0) ++b;
