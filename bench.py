@@ -43,8 +43,8 @@ def load_peaks():
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), float(d["bf16_tflops"]), "measured"
+    return 6650.0, 1400.0, 1590.0, "fallback"
 
 
 class ClockSampler:
@@ -176,6 +176,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=os.environ.get("TSID_BENCH_WORKLOAD", "C5"))
     ap.add_argument("--impl", default="tsid")
+    ap.add_argument("--path", default="sparse", choices=["auto", "sparse", "dense"],
+                    help="kernel path of the measured template (the dense tcgen05 variant needs a qualifying workload, e.g. C4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -213,7 +215,8 @@ def main():
     t1 = time.perf_counter()
     nnz = tpl.nnz
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
-    T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]
+    T = B.template_from_workload(tpl, path=want_path)
     torch.cuda.synchronize(dev)
     if rank == 0:
         sys.stderr.write("[bench] %s: generated %d entries in %.1f s, layout pass %.2f s, workspace %.2f GB\n" % (
@@ -269,7 +272,7 @@ def main():
     value = world * nnz * args.steps / (ms * 1e-3)
 
     # ---- roofline of the dominant kernel (the gather-reduce pass: two launches per step) ----------
-    peak, peak_kind = load_peaks()
+    peak, tf_sustained, tf_burst, peak_kind = load_peaks()
     nseg_row = w.m + nnz // 1024
     nseg_col = w.n + nnz // 1024
     b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col)
@@ -289,12 +292,27 @@ def main():
                 "step_alg_bytes": b_row + b_col + b_upd,
                 "step_frac": (b_row + b_col + b_upd) / (ms / args.steps * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+    if path == B.TSID_PATH_DENSE_TC:
+        # dense variant: the dominant kernel is the tcgen05 pass (two launches per step); algorithmic
+        # flops are the three GEMMs of the method, 6 m n k per step, i.e. 3 m n k per launch
+        flops_launch = 3.0 * w.m * w.n * w.k
+        tfl = flops_launch / (pass_ms * 1e-3) / 1e12 if pass_ms > 0 else 0.0
+        roofline = {"bound": "tensor", "kernel": "dense_pass_kernel (tcgen05; pass over R and pass over R^T)",
+                    "achieved": tfl, "peak": tf_sustained, "unit": "TFLOP/s", "frac": tfl / tf_sustained,
+                    "peak_source": "of %s (sustained bf16; burst %.1f)" % (peak_kind, tf_burst),
+                    "traffic": NCU_TRAFFIC_PER_LAUNCH.get(args.workload + "-dense"),
+                    "alg_flops_per_launch": flops_launch, "executed_flops_per_launch": 4.0 * w.m * w.n * w.k,
+                    "avg_launch_ms": pass_ms,
+                    "pass_R": {"ms": row_ms / max(1, nrec)}, "pass_RT": {"ms": col_ms / max(1, nrec)},
+                    "update": {"ms": upd_ms / max(1, nrec)},
+                    "step_frac": 6.0 * w.m * w.n * w.k / (ms / args.steps * 1e-3) / 1e12 / tf_sustained,
+                    "frac_of_nominal_2250": tfl / 2250.0}
 
     # ---- end to end: host buffers through tsid_fit_host ----------------------------------------------
     e2e = None
     if not args.no_e2e:
         epochs = args.e2e_epochs or w.epochs
-        cfg = B.make_config(w.m, w.n, w.k, nnz, prec, B.TSID_PATH_SPARSE, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
+        cfg = B.make_config(w.m, w.n, w.k, nnz, prec, want_path, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
         T.tsid_destroy()
         del T
         torch.cuda.empty_cache()
