@@ -14,8 +14,9 @@
 // owner CTA and a fixed summation order: no atomics, no partial buffers.  A 128x128x16 MMA with both
 // operands in shared memory reads 128 B per clock, the whole shared-memory bandwidth of an SM; keeping
 // E in TMEM removes its round trip through shared memory and halves what the second MMA reads there.
-// Shared-memory operands are K-major 128-byte-swizzled tiles, which is why transposed bf16 shadows
-// (k x rows) are kept next to the row-major ones.  Every mbarrier wait is bounded by a cycle budget; on
+// The Y tile (128 rows j x K columns, 128-byte-swizzled as TMA writes it) serves both products: K-major
+// as B of the first (contraction over the factor index) and MN-major as B of the second (contraction
+// over j), so no transposed copy of the factors exists.  Every mbarrier wait is bounded by a cycle budget; on
 // expiry the CTA raises FLAG_TIMEOUT, stops issuing, and still frees its TMEM before it returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -28,8 +29,7 @@ namespace tsid {
 
 struct DenseState {
   __half *R = nullptr, *RT = nullptr;              // [m*n], [n*m]; NaN = not observed
-  __nv_bfloat16 *PbT = nullptr, *QbT = nullptr;    // [k*m], [k*n]
-  CUtensorMap tmP, tmQ, tmPT, tmQT, tmR, tmRT;
+  CUtensorMap tmP, tmQ, tmR, tmRT;
 };
 
 namespace {
@@ -41,7 +41,7 @@ namespace {
   } while (0)
 
 constexpr int BLK = 128;                 // tile edge (rows of X per CTA, rows of Y per iteration)
-constexpr int NSTAGE = 2;                // stages of the Y / Y^T / R tiles
+constexpr int NSTAGE = 3;                // stages of the Y and R tiles
 constexpr long long WAIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz: bound of every wait
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -142,6 +142,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+// Descriptor of an MN-major operand read from the same kind of tile: rows of the tile are the K index
+// (8-row groups 1024 B apart), the 64 contiguous elements of a row are the MN index, and the next 64
+// MN elements live in the next 64-column block, `mn_block_bytes` further.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr, uint32_t mn_block_bytes) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_block_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
 // kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -152,19 +159,18 @@ struct Smem {
   static constexpr int XB = BLK * 128;            // one 64-column block of a 128-row tile: 16 KB
   static constexpr int X_BYTES = (K / 64) * XB;   // X block (128 x K bf16)
   static constexpr int Y_BYTES = (K / 64) * XB;   // Y block (128 x K bf16)
-  static constexpr int YTB = K * 128;             // one 64-column block of the K-row Y^T tile
-  static constexpr int YT_BYTES = 2 * YTB;        // Y^T block (K x 128 bf16)
   static constexpr int R_BYTES = 2 * XB;          // R tile (128 x 128 fp16)
-  static constexpr int STAGE_BYTES = Y_BYTES + YT_BYTES + R_BYTES;
+  static constexpr int STAGE_BYTES = Y_BYTES + R_BYTES;
   static constexpr int OFF_X = 0;
   static constexpr int OFF_Y = OFF_X + X_BYTES;
-  static constexpr int OFF_YT = OFF_Y + NSTAGE * Y_BYTES;
-  static constexpr int OFF_R = OFF_YT + NSTAGE * YT_BYTES;
+  static constexpr int OFF_R = OFF_Y + NSTAGE * Y_BYTES;
   static constexpr int OFF_BAR = OFF_R + NSTAGE * R_BYTES;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // barriers + slack for 1024-byte alignment
 };
 
-enum { B_XFULL = 0, B_QFULL = 1, B_QEMPTY = 3, B_SFULL = 5, B_SEMPTY = 7, B_EFULL = 9, B_EEMPTY = 11, B_GFULL = 13, B_COUNT = 14 };
+enum { B_XFULL = 0, B_QFULL = 1, B_QEMPTY = 1 + NSTAGE, B_SFULL = 1 + 2 * NSTAGE, B_SEMPTY = B_SFULL + 2, B_EFULL = B_SFULL + 4,
+       B_EEMPTY = B_SFULL + 6, B_GFULL = B_SFULL + 8, B_COUNT = B_SFULL + 9 };
+static_assert(B_COUNT * 8 <= 192, "barriers overlap the TMEM address slot");
 
 // TMEM columns (512 allocated): S tiles 0..127 and 128..255 (fp32), G block 256..383 (fp32, K used),
 // E tiles 384..447 and 448..511 (packed bf16: 64 columns hold 128 values per row).
@@ -178,14 +184,14 @@ constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_G = 256, TM_E0 = 384, TM_E1 = 448;
 template <int K>
 __global__ void __launch_bounds__(576, 1)
 dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-                  const __grid_constant__ CUtensorMap tmYT, const __grid_constant__ CUtensorMap tmR, int rows_y,
+                  const __grid_constant__ CUtensorMap tmR, int rows_y,
                   float *__restrict__ G, int32_t *__restrict__ flags) {
   using L = Smem<K>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;   // tiles need 1024-byte alignment
   unsigned char *smp = smem_dyn + (sm0 - s32(smem_dyn));
   const uint32_t bar0 = sm0 + L::OFF_BAR;
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smp + L::OFF_BAR + 128);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smp + L::OFF_BAR + 192);
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -201,7 +207,7 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(bar0 + 128u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(bar0 + 192u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -225,17 +231,15 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         mbar_expect_tx(bar(B_QFULL + st), L::STAGE_BYTES);
         for (int h = 0; h < K / 64; ++h)
           tma_load_2d(sm0 + L::OFF_Y + st * L::Y_BYTES + h * L::XB, &tmY, bar(B_QFULL + st), h * 64, jb * BLK);
-        for (int h = 0; h < 2; ++h) {
-          tma_load_2d(sm0 + L::OFF_YT + st * L::YT_BYTES + h * L::YTB, &tmYT, bar(B_QFULL + st), jb * BLK + h * 64, 0);
+        for (int h = 0; h < 2; ++h)
           tma_load_2d(sm0 + L::OFF_R + st * L::R_BYTES + h * L::XB, &tmR, bar(B_QFULL + st), jb * BLK + h * 64, ib * BLK);
-        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ---- MMA issuer -----------------------------------------------------------------------------
     if (lane == 0) {
-      constexpr uint32_t ID1 = idesc_bf16(BLK), ID2 = idesc_bf16(K);
+      constexpr uint32_t ID1 = idesc_bf16(BLK), ID2 = idesc_bf16(K) | (1u << 16);   // second product: B is MN-major
       auto mma1 = [&](int jb) -> bool {
         const int st = jb % NSTAGE, b = jb & 1;
         if (!mbar_wait(bar(B_QFULL + st), (jb / NSTAGE) & 1)) return false;
@@ -260,8 +264,9 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < BLK / 16; ++ks) {   // K of this product = the 128 columns j: 8 TMEM columns per step
-          const uint32_t offb = (ks / 4) * L::YTB + (ks % 4) * 32;
-          tc_mma_ts(tmG, tmE[b] + ks * 8, smem_desc(sm0 + L::OFF_YT + st * L::YT_BYTES + offb), ID2, (jb > 0 || ks > 0));
+          // B[K = j][N = l] is the Y tile itself read MN-major: 16 rows j per step = 2048 B
+          tc_mma_ts(tmG, tmE[b] + ks * 8, smem_desc_mn(sm0 + L::OFF_Y + st * L::Y_BYTES + ks * 2048, L::XB), ID2,
+                    (jb > 0 || ks > 0));
         }
         tc_commit(bar(B_EEMPTY + b));
         tc_commit(bar(B_QEMPTY + st));
@@ -277,7 +282,6 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int row = q * 32 + lane;          // row inside the tile
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t rrow0 = sm0 + L::OFF_R + h * L::XB + row * 128;   // this row in the R tile (block h)
-    static_assert(NSTAGE == 2, "a team owns one stage, one S buffer and one E buffer");
     for (int jb = team; jb < NJ && ok; jb += 2) {
       const int b = jb & 1, st = jb % NSTAGE;
       ok = mbar_wait(bar(B_QFULL + st), (jb / NSTAGE) & 1);                   // R tile has landed
@@ -371,22 +375,6 @@ __global__ void scatter_dense_kernel(const int64_t *__restrict__ row_ptr, const 
   }
 }
 
-// out[k][rows] = in[rows][k]   (bf16)
-__global__ void transpose_bf16_kernel(const __nv_bfloat16 *__restrict__ in, __nv_bfloat16 *__restrict__ out, int rows,
-                                      int k) {
-  __shared__ __nv_bfloat16 t[32][33];
-  const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
-  for (int y = threadIdx.y; y < 32; y += blockDim.y) {
-    const int r = r0 + y, c = c0 + threadIdx.x;
-    if (r < rows && c < k) t[y][threadIdx.x] = in[(size_t)r * k + c];
-  }
-  __syncthreads();
-  for (int y = threadIdx.y; y < 32; y += blockDim.y) {
-    const int c = c0 + y, r = r0 + threadIdx.x;
-    if (r < rows && c < k) out[(size_t)c * rows + r] = t[threadIdx.x][y];
-  }
-}
-
 typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -412,11 +400,11 @@ cudaError_t make_map(CUtensorMap *tm, CUtensorMapDataType dt, void *base, uint64
 }
 
 template <int K>
-cudaError_t launch_dense_pass(cudaStream_t st, const CUtensorMap &tmX, const CUtensorMap &tmY, const CUtensorMap &tmYT,
+cudaError_t launch_dense_pass(cudaStream_t st, const CUtensorMap &tmX, const CUtensorMap &tmY,
                               const CUtensorMap &tmR, int rows_x, int rows_y, float *G, int32_t *flags) {
   auto kern = dense_pass_kernel<K>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<K>::TOTAL));
-  kern<<<rows_x / BLK, 576, Smem<K>::TOTAL, st>>>(tmX, tmY, tmYT, tmR, rows_y, G, flags);
+  kern<<<rows_x / BLK, 576, Smem<K>::TOTAL, st>>>(tmX, tmY, tmR, rows_y, G, flags);
   return cudaGetLastError();
 }
 
@@ -431,8 +419,7 @@ void dense_carve(tsid_template *t, const tsid_config_t &c, Carver &cv) {
   DenseState *d = t->dense;
   const size_t mn = (size_t)c.m * c.n;
   __half *R = cv.take<__half>(mn), *RT = cv.take<__half>(mn);
-  __nv_bfloat16 *PbT = cv.take<__nv_bfloat16>((size_t)c.m * c.k), *QbT = cv.take<__nv_bfloat16>((size_t)c.n * c.k);
-  if (d) { d->R = R; d->RT = RT; d->PbT = PbT; d->QbT = QbT; }
+  if (d) { d->R = R; d->RT = RT; }
 }
 
 DenseState *dense_new() { return new (std::nothrow) DenseState; }
@@ -453,8 +440,6 @@ cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag) {
   const CUtensorMapDataType BF = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, HF = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
   CK(make_map(&d->tmP, BF, t->rowside.shadow, c.m, c.k, BLK));
   CK(make_map(&d->tmQ, BF, t->colside.shadow, c.n, c.k, BLK));
-  CK(make_map(&d->tmPT, BF, d->PbT, c.k, c.m, c.k));
-  CK(make_map(&d->tmQT, BF, d->QbT, c.k, c.n, c.k));
   CK(make_map(&d->tmR, HF, d->R, c.m, c.n, BLK));
   CK(make_map(&d->tmRT, HF, d->RT, c.n, c.m, BLK));
   return cudaSuccess;
@@ -465,19 +450,15 @@ cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ) {
   DenseState *d = t->dense;
   const tsid_config_t &c = t->cfg;
   cudaStream_t st = t->stream;
-  dim3 tb(32, 8);
-  transpose_bf16_kernel<<<dim3((c.m + 31) / 32, (c.k + 31) / 32), tb, 0, st>>>(t->rowside.shadow, d->PbT, c.m, c.k);
-  transpose_bf16_kernel<<<dim3((c.n + 31) / 32, (c.k + 31) / 32), tb, 0, st>>>(t->colside.shadow, d->QbT, c.n, c.k);
-  CK(cudaGetLastError());
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW0], st);
-  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmP, d->tmQ, d->tmQT, d->tmR, c.m, c.n, GP, t->flags));
-  else CK(launch_dense_pass<64>(st, d->tmP, d->tmQ, d->tmQT, d->tmR, c.m, c.n, GP, t->flags));
+  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmP, d->tmQ, d->tmR, c.m, c.n, GP, t->flags));
+  else CK(launch_dense_pass<64>(st, d->tmP, d->tmQ, d->tmR, c.m, c.n, GP, t->flags));
   if (t->prof.on && t->prof.nsteps < kProfSteps) {
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW1], st);
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL0], st);
   }
-  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmQ, d->tmP, d->tmPT, d->tmRT, c.n, c.m, GQ, t->flags));
-  else CK(launch_dense_pass<64>(st, d->tmQ, d->tmP, d->tmPT, d->tmRT, c.n, c.m, GQ, t->flags));
+  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmQ, d->tmP, d->tmRT, c.n, c.m, GQ, t->flags));
+  else CK(launch_dense_pass<64>(st, d->tmQ, d->tmP, d->tmRT, c.n, c.m, GQ, t->flags));
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL1], st);
   return cudaSuccess;
 }

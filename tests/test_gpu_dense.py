@@ -80,7 +80,7 @@ def test_dense_trajectory_rmse_and_determinism():
     r, c, v = np_coo(tpl)
     P0, Q0 = tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy()
     T = B.template_from_workload(tpl)             # AUTO: dense at 30 % density
-    assert T.tsid_get_info() == (B.TSID_PATH_DENSE_TC, 6)
+    assert T.tsid_get_info() == (B.TSID_PATH_DENSE_TC, 4)
     P, Q = tpl.P0.clone(), tpl.Q0.clone()
     hist = np.array(T.tsid_fit(P, Q, w.epochs, loss_every=1))
     _, _, ref_hist = oracle.fit(w.m, w.n, w.k, r, c, v, P0, Q0, w.epochs, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
