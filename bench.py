@@ -97,6 +97,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x, dist, device):
+    """The slowest rank's time (replicas run independently; the job is as slow as its slowest rank)."""
+    if dist is None:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(world, units_per_rank_step, steps, seconds):
+    """Whole-job throughput: every rank processed units_per_rank_step * steps units in `seconds`."""
+    return world * units_per_rank_step * steps / seconds
+
+
 def alg_bytes(w, nnz, nseg_row, nseg_col):
     """Algorithmic bytes of one launch of each kernel of a step ("Roofline")."""
     b = 2 if w.precision == "bf16" else 4
@@ -143,7 +157,7 @@ def run_reference(args, W):
     print(json.dumps(line))
 
 
-def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=15.0):
+def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=20.0):
     """Times the oracle on a prefix of the template's (row-sorted) COO entries with the full factor
     matrices; sized from a short calibration run so that it takes about budget_s seconds."""
     import numpy as np
@@ -265,11 +279,8 @@ def main():
     T.tsid_set_profiling(False)
     T.tsid_check()
 
-    if dist is not None:
-        tms = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
-    value = world * nnz * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, dist, dev)
+    value = aggregate_value(world, nnz, args.steps, ms * 1e-3)
 
     # ---- roofline of the dominant kernel (the gather-reduce pass: two launches per step) ----------
     peak, tf_sustained, tf_burst, peak_kind = load_peaks()
@@ -331,10 +342,7 @@ def main():
             torch.cuda.synchronize(dev)
             if rep > 0:   # the first call warms the pinned pages and the allocator
                 t_e2e += time.perf_counter() - t0
-        if dist is not None:
-            tt = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            t_e2e = float(tt.item())
+        t_e2e = max_over_ranks(t_e2e, dist, dev)
         h2d = nnz * 12 + (w.m + w.n) * w.k * 4
         d2h = (w.m + w.n) * w.k * 4
         e2e = {"value": world * nnz * epochs * reps / t_e2e, "unit": UNIT,
