@@ -33,8 +33,9 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the gather-reduce pass kernel
 # (average of the row pass and the column pass), from the ncu summaries under profiles/.
 NCU_TRAFFIC_PER_LAUNCH = {
-    "C5": 91.79e9,   # profiles/pass_kernel_C5_launches_dram.md: row 76.95 GB, column 106.63 GB
-    "C3": 0.882e9,   # profiles/pass_kernel_C3_ncu_full.md: row 0.892 GB, column 0.872 GB
+    "C5": 92.14e9,        # profiles/step_kernels_C5_launches_dram.md: row 77.23 GB, column 107.06 GB
+    "C3": 0.865e9,        # profiles/pass_staged_kernel_C3_ncu.md
+    "C4-dense": 0.551e9,  # profiles/dense_pass_kernel_C4_ncu.md: the fp16 R matrix once per launch
 }
 
 
@@ -157,7 +158,7 @@ def run_reference(args, W):
     print(json.dumps(line))
 
 
-def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=20.0):
+def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=25.0):
     """Times the oracle on a prefix of the template's (row-sorted) COO entries with the full factor
     matrices; sized from a short calibration run so that it takes about budget_s seconds."""
     import numpy as np
@@ -301,6 +302,7 @@ def main():
                 "update": {"ms": upd_ms / max(1, nrec), "alg_bytes": b_upd,
                            "gbs": b_upd / (upd_ms / max(1, nrec) * 1e-3) / 1e9 if upd_ms else None},
                 "step_alg_bytes": b_row + b_col + b_upd,
+                "step_compulsory_bytes": nnz * 16 + (w.m + w.n) * w.k * 20,   # perfect cache: streams + factors once
                 "step_frac": (b_row + b_col + b_upd) / (ms / args.steps * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     if path == B.TSID_PATH_DENSE_TC:
