@@ -184,6 +184,46 @@ def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=25.0):
                       "%.1f s" % (count, nnz, m_used - 1, w.n, t)}
 
 
+def measure_sampling(args, w, tpl, B, dev):
+    """Times tsid_sample_template (alpha = 0.5) on the workload's COO triples taken as the full matrix."""
+    import ctypes as C
+    nnz = tpl.nnz
+    alpha, seed = 0.5, 12345
+    need = C.c_size_t(0)
+    B.lib().tsid_sample_workspace_bytes(w.n, nnz, C.byref(need))
+    ws = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    base = (ws.data_ptr() + 255) & ~255
+    colmap = torch.empty(w.n, dtype=torch.int32, device=dev)
+    ro, co = torch.empty(nnz, dtype=torch.int32, device=dev), torch.empty(nnz, dtype=torch.int32, device=dev)
+    vo = torch.empty(nnz, dtype=torch.float32, device=dev)
+    d, kept = C.c_int32(0), C.c_int64(0)
+    stream = torch.cuda.current_stream(dev)
+
+    def call():
+        st = B.lib().tsid_sample_template(w.m, w.n, nnz, alpha, seed, tpl.rows.data_ptr(), tpl.cols.data_ptr(),
+                                          tpl.vals.data_ptr(), stream.cuda_stream, base, need.value, colmap.data_ptr(),
+                                          ro.data_ptr(), co.data_ptr(), vo.data_ptr(), C.byref(d), C.byref(kept))
+        assert st == B.TSID_OK, st
+    for _ in range(args.warmup):
+        call()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        call()
+    b.record(stream)
+    torch.cuda.synchronize(dev)
+    ms = a.elapsed_time(b) / args.steps
+    peak = load_peaks()[0]
+    # per entry: column read for the keep flag (4) + flag write, scan read and write (12) + triple read (12)
+    # + position read (8); per kept entry: triple write (12)
+    alg = nnz * 36 + kept.value * 12
+    print(json.dumps({"metric": "matrix entries sampled/sec", "value": nnz / (ms * 1e-3), "unit": "entries/s",
+                      "ms_per_call": ms, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "config": {"workload": w.name, "alpha": alpha, "d": d.value, "kept": kept.value},
+                      "roofline": {"bound": "hbm", "achieved": alg / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": alg / (ms * 1e-3) / 1e9 / peak, "alg_bytes": alg}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -193,6 +233,8 @@ def main():
     ap.add_argument("--impl", default="tsid")
     ap.add_argument("--path", default="sparse", choices=["auto", "sparse", "dense"],
                     help="kernel path of the measured template (the dense tcgen05 variant needs a qualifying workload, e.g. C4)")
+    ap.add_argument("--measure", default="step", choices=["step", "sample"],
+                    help="step: the gradient step (default); sample: tsid_sample_template on the workload's COO")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -229,6 +271,9 @@ def main():
     torch.cuda.synchronize(dev)
     t1 = time.perf_counter()
     nnz = tpl.nnz
+    if args.measure == "sample":
+        measure_sampling(args, w, tpl, B, dev)
+        return
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
     want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]
     T = B.template_from_workload(tpl, path=want_path)

@@ -177,6 +177,28 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
  * tsid_grad_step launches. */
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
 
+/* Template sampling (Sec. 5.1, "Sampling the TSID Template Submatrix"): the step before the
+ * factorization.  Chooses d = ceil(alpha n) of the n columns uniformly at random without replacement
+ * and extracts the template R* = { r_ij : j chosen, (i,j) in Omega } as COO triples with the chosen
+ * columns re-indexed 0..d-1 in ascending order of their original index (rows unchanged, kept entries
+ * in input order), ready for tsid_template_create with n = d.  The draw is counter-based and
+ * reproducible: column j gets the key SplitMix64(seed + (j+1) * 0x9E3779B97F4A7C15) and the d columns
+ * with the smallest (key, j) are taken.
+ *   - d_rows, d_cols, d_vals: DEVICE, the COO triples of the full matrix (m x n, nnz entries, any order).
+ *   - d_colmap: DEVICE int32[n], out: new index of each column, or -1 if it is not in the template.
+ *   - d_rows_out, d_cols_out, d_vals_out: DEVICE, capacity nnz each, out: the template's triples.
+ *   - h_d_out, h_nnz_out: HOST, out: d and the number of template entries.
+ *   - workspace: DEVICE, 256-byte aligned, tsid_sample_workspace_bytes(n, nnz) bytes; nothing is allocated.
+ * 0 < alpha <= 1.  Work is enqueued on `stream`; the call synchronises it before writing the host outputs.
+ * Errors: TSID_ERR_INVALID_ARG, TSID_ERR_OOM (workspace too small), TSID_ERR_INDEX_RANGE (a column index
+ * outside [0, n)), TSID_ERR_CUDA. */
+tsid_status_t tsid_sample_workspace_bytes(int32_t n, int64_t nnz, size_t *h_bytes_out);
+tsid_status_t tsid_sample_template(int32_t m, int32_t n, int64_t nnz, double alpha, uint64_t seed,
+                                   const int32_t *d_rows, const int32_t *d_cols, const float *d_vals,
+                                   void *stream, void *workspace, size_t workspace_bytes,
+                                   int32_t *d_colmap, int32_t *d_rows_out, int32_t *d_cols_out,
+                                   float *d_vals_out, int32_t *h_d_out, int64_t *h_nnz_out);
+
 /* Per-kernel timing for benchmarks.  tsid_set_profiling(t, 1) makes every following step record
  * CUDA events on the template's stream right before and after its row pass, its column pass
  * and its update kernel (at most 256 steps are kept); 0 turns it off and frees the events.

@@ -159,3 +159,25 @@ def layout(m, n, rows, cols, vals) -> Layout:
                     _p(out.col_ptr, C.c_int64), _p(out.row_idx, C.c_int32), _p(out.val_csc, C.c_float),
                     _p(out.perm, C.c_uint32))
     return out
+
+
+def splitmix64_at(seed: int, index1: int) -> int:
+    f = _L().orc_splitmix64_at
+    f.restype = C.c_uint64
+    f.argtypes = [C.c_uint64, C.c_uint64]
+    return int(f(seed, index1))
+
+
+def sample_template(m, n, rows, cols, vals, alpha, seed):
+    """Returns (colmap int32[n], rows', cols', vals', d)."""
+    rows, cols, vals = _coo(rows, cols, vals)
+    nnz = rows.shape[0]
+    colmap = np.empty(n, np.int32)
+    ro, co, vo = np.empty(nnz, np.int32), np.empty(nnz, np.int32), np.empty(nnz, np.float32)
+    d = C.c_int32(0); kept = C.c_int64(0)
+    _L().orc_sample_template(C.c_int32(m), C.c_int32(n), C.c_int64(nnz), C.c_double(alpha), C.c_uint64(seed),
+                             _p(rows, C.c_int32), _p(cols, C.c_int32), _p(vals, C.c_float),
+                             _p(colmap, C.c_int32), _p(ro, C.c_int32), _p(co, C.c_int32), _p(vo, C.c_float),
+                             C.byref(d), C.byref(kept))
+    k = kept.value
+    return colmap, ro[:k].copy(), co[:k].copy(), vo[:k].copy(), d.value

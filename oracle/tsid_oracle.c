@@ -254,3 +254,53 @@ void orc_layout(int32_t m, int32_t n, int64_t nnz,
   free(keys);
   free(csr_pos);
 }
+
+/* ---- template sampling (Sec. 5.1, "Sampling the TSID Template Submatrix") ---------------------
+ * C = d = ceil(alpha n) columns drawn uniformly at random without replacement; the template keeps
+ * the observed entries whose column is in C.  Readings: the draw is made reproducible by giving
+ * column j the key SplitMix64(seed + (j+1) * 0x9E3779B97F4A7C15), i.e. the (j+1)-th output of the
+ * SplitMix64 generator seeded with `seed`, and taking the d columns with the smallest (key, j)
+ * (a uniformly random d-subset); the chosen columns are re-indexed 0..d-1 in ascending order of
+ * their original index; rows are unchanged; kept entries stay in input order.
+ * Pins: published SplitMix64 outputs; |C| = d; brute-force membership; inclusion frequency. */
+uint64_t orc_splitmix64_at(uint64_t seed, uint64_t index1) {
+  uint64_t z = seed + index1 * 0x9E3779B97F4A7C15ULL;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+
+typedef struct { uint64_t key; int32_t col; } orc_colkey_t;
+
+static int colkey_cmp(const void *x, const void *y) {
+  const orc_colkey_t *u = (const orc_colkey_t *)x, *v = (const orc_colkey_t *)y;
+  if (u->key != v->key) return (u->key < v->key) ? -1 : 1;
+  if (u->col != v->col) return (u->col < v->col) ? -1 : 1;
+  return 0;
+}
+
+/* colmap[n] receives the new column index or -1; the *_out arrays need capacity nnz.
+ * Returns d through d_out and the number of kept entries through nnz_out. */
+void orc_sample_template(int32_t m, int32_t n, int64_t nnz, double alpha, uint64_t seed,
+                         const int32_t *rows, const int32_t *cols, const float *vals,
+                         int32_t *colmap, int32_t *rows_out, int32_t *cols_out, float *vals_out,
+                         int32_t *d_out, int64_t *nnz_out) {
+  (void)m;
+  double dd = ceil(alpha * (double)n);
+  int32_t d = dd < 1.0 ? 1 : (dd > (double)n ? n : (int32_t)dd);
+  orc_colkey_t *ck = (orc_colkey_t *)malloc(sizeof(orc_colkey_t) * (size_t)n);
+  for (int32_t j = 0; j < n; ++j) { ck[j].key = orc_splitmix64_at(seed, (uint64_t)j + 1); ck[j].col = j; }
+  qsort(ck, (size_t)n, sizeof(orc_colkey_t), colkey_cmp);
+  for (int32_t j = 0; j < n; ++j) colmap[j] = -1;
+  for (int32_t q = 0; q < d; ++q) colmap[ck[q].col] = 0;      /* chosen */
+  int32_t next = 0;
+  for (int32_t j = 0; j < n; ++j) if (colmap[j] == 0) colmap[j] = next++;
+  int64_t o = 0;
+  for (int64_t t = 0; t < nnz; ++t) {
+    int32_t c = colmap[cols[t]];
+    if (c >= 0) { rows_out[o] = rows[t]; cols_out[o] = c; vals_out[o] = vals[t]; ++o; }
+  }
+  *d_out = d;
+  *nnz_out = o;
+  free(ck);
+}

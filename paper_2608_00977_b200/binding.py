@@ -31,7 +31,7 @@ TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
 EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",
            "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
-           "tsid_get_pass_times", "tsid_sse_noalloc"]
+           "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template"]
 
 
 class TsidConfig(C.Structure):
@@ -78,6 +78,9 @@ def lib():
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
         L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
         L.tsid_sse_noalloc.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
+        L.tsid_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
+        L.tsid_sample_template.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_uint64, vp, vp, vp, vp, vp,
+                                           C.c_size_t, vp, vp, vp, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
         L.tsid_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name != "tsid_last_error":
@@ -289,6 +292,35 @@ def tsid_sse_noalloc(m, n, k, rows, cols, vals, P, Q, out, stream=None):
                                     Q.data_ptr(), stream.cuda_stream, out.data_ptr())
     if st != TSID_OK:
         raise TsidError(st, "tsid_sse_noalloc refused or failed")
+
+
+def tsid_sample_template(m, n, rows, cols, vals, alpha, seed, stream=None):
+    """Column sampling + template extraction.  Returns (colmap int32[n], rows', cols', vals', d) as CUDA
+    tensors (the triples trimmed to the number of template entries)."""
+    nnz = int(rows.numel())
+    _check_tensor(rows, torch.int32, nnz, "rows")
+    _check_tensor(cols, torch.int32, nnz, "cols")
+    _check_tensor(vals, torch.float32, nnz, "vals")
+    dev = rows.device
+    need = C.c_size_t(0)
+    st = lib().tsid_sample_workspace_bytes(n, nnz, C.byref(need))
+    if st != TSID_OK:
+        raise TsidError(st, "tsid_sample_workspace_bytes")
+    ws = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    base = (ws.data_ptr() + 255) & ~255
+    colmap = torch.empty(n, dtype=torch.int32, device=dev)
+    ro, co = torch.empty(max(nnz, 1), dtype=torch.int32, device=dev), torch.empty(max(nnz, 1), dtype=torch.int32, device=dev)
+    vo = torch.empty(max(nnz, 1), dtype=torch.float32, device=dev)
+    d, kept = C.c_int32(0), C.c_int64(0)
+    stream = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        st = lib().tsid_sample_template(m, n, nnz, float(alpha), int(seed), rows.data_ptr(), cols.data_ptr(),
+                                        vals.data_ptr(), stream.cuda_stream, base, need.value, colmap.data_ptr(),
+                                        ro.data_ptr(), co.data_ptr(), vo.data_ptr(), C.byref(d), C.byref(kept))
+    if st != TSID_OK:
+        raise TsidError(st, "tsid_sample_template")
+    k = kept.value
+    return colmap, ro[:k], co[:k], vo[:k], d.value
 
 
 def template_from_workload(tpl, path=TSID_PATH_AUTO, flags=0, precision=None) -> Template:

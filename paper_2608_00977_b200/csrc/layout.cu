@@ -418,4 +418,13 @@ cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutSc
   return cudaStreamSynchronize(st);
 }
 
+// The sort and the scan, for the other translation units (template sampling).
+cudaError_t sort_pairs_u32(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits, LayoutScratch &s,
+                           cudaStream_t st, uint32_t **kres, uint32_t **vres) {
+  return radix_sort_pairs(kin, vin, n, nbits, s, st, kres, vres);
+}
+cudaError_t scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch &s, cudaStream_t st) {
+  return exclusive_scan_u32(in, out, n, s, st);
+}
+
 }  // namespace tsid

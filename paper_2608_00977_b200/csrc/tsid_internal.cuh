@@ -113,6 +113,12 @@ constexpr int kScanBlocksMax = 1 << 20;
 cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols,
                          const float *d_vals, LayoutScratch &s, int32_t h_flags[FLAG_COUNT]);
 cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutScratch &s);
+// stable LSD radix sort of (key, payload) pairs on key bits [0, nbits) (vin == nullptr: payload = position);
+// ping-pongs between (s.kA, s.vA) and (s.kB, s.vB), the input must not live in kA / vA
+cudaError_t sort_pairs_u32(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits, LayoutScratch &s,
+                           cudaStream_t st, uint32_t **kres, uint32_t **vres);
+// out[0..n) = exclusive scan of in[0..n), out[n] = total; in[n] must be 0; in may alias out
+cudaError_t scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch &s, cudaStream_t st);
 
 // sparse passes (sparse.cu)
 cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);
