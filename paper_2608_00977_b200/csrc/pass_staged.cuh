@@ -45,7 +45,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // per SM) measured 9 % faster than the unconstrained 101; tighter caps spill and lose.
 template <int KP, bool BF16>
 struct StagedMinBlocks {
-  static constexpr int value = (KP == 128 && BF16) ? 18 : 1;
+  static constexpr int value = KP <= 64 ? 32 : (KP == 128 ? 18 : 1);
 };
 
 template <int KP, bool BF16, int NST, int ROWS>
