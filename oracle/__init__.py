@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tsid_oracle.c")
 _LIB = os.path.join(_HERE, "libtsid_oracle.so")
 
-CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD = 0, 1, 2
+CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD, CLIP_ASYM_ENTRY = 0, 1, 2, 3
 NORM_NONE, NORM_COUNT = 0, 1
 
 

@@ -28,7 +28,14 @@
  *     CLIP_ASYM_STEP: D <- min(max(xi,-D), D)   (caps increases at eta*xi);
  *     CLIP_ASYM_GRAD: the same formula applied to the loss gradient g = -D,
  *     then the step is -eta * clip(g);
- *   - both factor updates use the same residuals (Jacobi, simultaneous).
+ *   - both factor updates use the same residuals (Jacobi, simultaneous);
+ *   - CLIP_ASYM_ENTRY is the equation of Sec. 5.3 taken literally, entry by entry: every
+ *     observed (i,j) contributes its own clipped direction
+ *         c_ij = min(max(xi, -d_ij), d_ij),  d_ij = 2 e_ij q_j - 2 lambda p_i   (for p_i),
+ *     the contributions of a factor row are added and divided by s (Eq. 9's 1/n), and the
+ *     row moves by eta times that.  Here the regulariser sits inside every entry's term, and a
+ *     row without entries does not move.  The "gradient sums" returned in this mode are the
+ *     sums of the c_ij.
  *
  * Pins: every function below is pinned by tests marked "not gpu" (hand-worked
  * 3x2 and 8x6 examples stored as golden text, finite differences of the loss,
@@ -44,7 +51,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORC_CLIP_NONE = 0, ORC_CLIP_ASYM_STEP = 1, ORC_CLIP_ASYM_GRAD = 2 };
+enum { ORC_CLIP_NONE = 0, ORC_CLIP_ASYM_STEP = 1, ORC_CLIP_ASYM_GRAD = 2, ORC_CLIP_ASYM_ENTRY = 3 };
 enum { ORC_NORM_NONE = 0, ORC_NORM_COUNT = 1 };
 
 /* Round a float to the nearest bfloat16 (ties to even) and return it as float.
@@ -150,9 +157,38 @@ void orc_grad_step(int32_t m, int32_t n, int32_t k, int64_t nnz,
                    float *P_new, float *Q_new) {
   int64_t *cntP = (int64_t *)malloc(sizeof(int64_t) * (size_t)(m > 0 ? m : 1));
   int64_t *cntQ = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n > 0 ? n : 1));
-  orc_grad_sums(m, n, k, nnz, rows, cols, vals, P, Q, bf16_emulate, GP, GQ, cntP, cntQ);
-  direction(m, k, GP, cntP, P, lambda, xi, clip, norm_p, DP);
-  direction(n, k, GQ, cntQ, Q, lambda, xi, clip, norm_q, DQ);
+  if (clip == ORC_CLIP_ASYM_ENTRY) {
+    memset(GP, 0, sizeof(double) * (size_t)m * k);
+    memset(GQ, 0, sizeof(double) * (size_t)n * k);
+    memset(cntP, 0, sizeof(int64_t) * (size_t)(m > 0 ? m : 1));
+    memset(cntQ, 0, sizeof(int64_t) * (size_t)(n > 0 ? n : 1));
+    for (int64_t t = 0; t < nnz; ++t) {
+      int64_t i = rows[t], j = cols[t];
+      double dot = 0.0;
+      for (int32_t l = 0; l < k; ++l)
+        dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
+      double e = (double)vals[t] - dot;
+      for (int32_t l = 0; l < k; ++l) {
+        double pv = read_factor(P, i * k + l, bf16_emulate), qv = read_factor(Q, j * k + l, bf16_emulate);
+        GP[i * k + l] += orc_clip_nested(2.0 * e * qv - 2.0 * lambda * pv, xi);
+        GQ[j * k + l] += orc_clip_nested(2.0 * e * pv - 2.0 * lambda * qv, xi);
+      }
+      cntP[i] += 1;
+      cntQ[j] += 1;
+    }
+    for (int64_t r = 0; r < m; ++r) {
+      double sc = (norm_p == ORC_NORM_COUNT && cntP[r] > 1) ? (double)cntP[r] : 1.0;
+      for (int32_t l = 0; l < k; ++l) DP[r * k + l] = GP[r * k + l] / sc;
+    }
+    for (int64_t r = 0; r < n; ++r) {
+      double sc = (norm_q == ORC_NORM_COUNT && cntQ[r] > 1) ? (double)cntQ[r] : 1.0;
+      for (int32_t l = 0; l < k; ++l) DQ[r * k + l] = GQ[r * k + l] / sc;
+    }
+  } else {
+    orc_grad_sums(m, n, k, nnz, rows, cols, vals, P, Q, bf16_emulate, GP, GQ, cntP, cntQ);
+    direction(m, k, GP, cntP, P, lambda, xi, clip, norm_p, DP);
+    direction(n, k, GQ, cntQ, Q, lambda, xi, clip, norm_q, DQ);
+  }
   for (int64_t a = 0; a < (int64_t)m * k; ++a) P_new[a] = (float)((double)P[a] + eta * DP[a]);
   for (int64_t a = 0; a < (int64_t)n * k; ++a) Q_new[a] = (float)((double)Q[a] + eta * DQ[a]);
   free(cntP);

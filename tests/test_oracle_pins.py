@@ -88,6 +88,24 @@ def test_worked_example_directions(golden_3x2):
     assert np.array_equal(st.DQ, _arr(g, "DQ_count", (n, k)))
 
 
+def test_worked_example_entrywise_clip(golden_3x2):
+    """Sec. 5.3 taken entry by entry: clipped per-entry directions, summed, divided by the count on the q side."""
+    g = golden_3x2
+    m, n, k, rows, cols, vals, P, Q = _inst(g)
+    eta, lam, xi = g["eta"][0], g["lambda"][0], g["xi"][0]
+    st = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, eta, lam, xi, oracle.CLIP_ASYM_ENTRY, 0, 0)
+    assert np.array_equal(st.GP, _arr(g, "GP_entry", (m, k))) and np.array_equal(st.GQ, _arr(g, "GQ_entry", (n, k)))
+    np.testing.assert_allclose(st.P, _arr(g, "P1_entry_none", (m, k)), rtol=0, atol=1e-7)
+    np.testing.assert_allclose(st.Q, _arr(g, "Q1_entry_none", (n, k)), rtol=0, atol=1e-7)
+    st = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, eta, lam, xi, oracle.CLIP_ASYM_ENTRY, 0, 1)
+    np.testing.assert_allclose(st.P, _arr(g, "P1_entry_none", (m, k)), rtol=0, atol=1e-7)
+    np.testing.assert_allclose(st.Q, _arr(g, "Q1_entry_count", (n, k)), rtol=0, atol=1e-7)
+    # with a threshold that never bites and lambda = 0 it is the plain summed direction 2 G / s
+    big = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, eta, 0.0, 1e30, oracle.CLIP_ASYM_ENTRY, 1, 1)
+    ref = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, eta, 0.0, 1e30, oracle.CLIP_NONE, 1, 1)
+    np.testing.assert_allclose(big.DP, ref.DP, rtol=1e-15) and np.testing.assert_allclose(big.DQ, ref.DQ, rtol=1e-15)
+
+
 def test_worked_example_layout(golden_3x2):
     g = golden_3x2
     lay = oracle.layout(3, 2, _arr(g, "shuf_rows", dtype=np.int32), _arr(g, "shuf_cols", dtype=np.int32),
@@ -106,6 +124,11 @@ def _brute_force_dense(m, n, k, mask, R, P, Q, eta, lam, xi, clip, norm_p, norm_
     GQ = [[sum(E[i][j] * P[i][l] for i in range(m)) for l in range(k)] for j in range(n)]
     cr = [sum(mask[i]) for i in range(m)]
     cc = [sum(mask[i][j] for i in range(m)) for j in range(n)]
+    if clip == oracle.CLIP_ASYM_ENTRY:   # every observed cell adds its own clipped direction
+        GP = [[sum(min(2 * E[i][j] * Q[j][l] - 2 * lam * P[i][l], xi) for j in range(n) if mask[i][j])
+               for l in range(k)] for i in range(m)]
+        GQ = [[sum(min(2 * E[i][j] * P[i][l] - 2 * lam * Q[j][l], xi) for i in range(m) if mask[i][j])
+               for l in range(k)] for j in range(n)]
 
     def upd(X, G, cnt, norm):
         out = []
@@ -113,6 +136,9 @@ def _brute_force_dense(m, n, k, mask, R, P, Q, eta, lam, xi, clip, norm_p, norm_
             s = max(1, cnt[r]) if norm else 1
             new = []
             for l, x in enumerate(row):
+                if clip == oracle.CLIP_ASYM_ENTRY:
+                    new.append(x + eta * G[r][l] / s)
+                    continue
                 d = 2 * G[r][l] / s - 2 * lam * x
                 if clip == oracle.CLIP_ASYM_STEP:
                     d = min(d, xi)          # the verbal rule: positive values above xi become xi
@@ -127,7 +153,7 @@ def _brute_force_dense(m, n, k, mask, R, P, Q, eta, lam, xi, clip, norm_p, norm_
 
 
 @pytest.mark.parametrize("clip,norm_p,norm_q", list(itertools.product(
-    [oracle.CLIP_NONE, oracle.CLIP_ASYM_STEP, oracle.CLIP_ASYM_GRAD], [0, 1], [0, 1])))
+    [oracle.CLIP_NONE, oracle.CLIP_ASYM_STEP, oracle.CLIP_ASYM_GRAD, oracle.CLIP_ASYM_ENTRY], [0, 1], [0, 1])))
 def test_8x6_rank2_brute_force(clip, norm_p, norm_q):
     g = read_golden("rank2_8x6.txt")
     m, n, k = 8, 6, 2
