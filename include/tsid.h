@@ -78,8 +78,16 @@ typedef enum { TSID_PATH_AUTO = 0, TSID_PATH_SPARSE = 1, TSID_PATH_DENSE_TC = 2 
 
 /* Sec. 5.3.  ASYM_STEP (default reading): D <- min(max(xi, -D), D) = min(D, xi): increases
  * of a coordinate are capped at eta*xi, decreases are free.  ASYM_GRAD: the same formula
- * applied to the loss gradient g = -D, i.e. D <- max(D, -xi). */
-typedef enum { TSID_CLIP_NONE = 0, TSID_CLIP_ASYM_STEP = 1, TSID_CLIP_ASYM_GRAD = 2 } tsid_clip_t;
+ * applied to the loss gradient g = -D, i.e. D <- max(D, -xi).  ASYM_ENTRY: the equation of
+ * Sec. 5.3 taken entry by entry, as printed: every observed (i,j) contributes its own clipped
+ * direction c_ij = min(2 e_ij q_j - 2 lambda p_i, xi) (for p_i; symmetrically for q_j), the
+ * contributions of a factor row are added, divided by s (Eq. 9's 1/n) and applied with eta.
+ * In this mode the regulariser sits inside every entry's term, a row without entries does not
+ * move, the values read are those of the template's precision, and d_gradP / d_gradQ receive
+ * the sums of the c_ij.  Sparse path only. */
+typedef enum {
+  TSID_CLIP_NONE = 0, TSID_CLIP_ASYM_STEP = 1, TSID_CLIP_ASYM_GRAD = 2, TSID_CLIP_ASYM_ENTRY = 3
+} tsid_clip_t;
 
 /* Eq. 9's 1/n factor: divide the summed gradient of a factor row by the number of
  * observed entries that contribute to it (COUNT) or not at all (NONE). */

@@ -23,7 +23,7 @@ TSID_ERR_TOO_LARGE = 9
  TSID_ERR_CUDA, TSID_ERR_UNSUPPORTED, TSID_ERR_NONFINITE) = range(1, 9)
 TSID_F32, TSID_BF16_SHADOW = 0, 1
 TSID_PATH_AUTO, TSID_PATH_SPARSE, TSID_PATH_DENSE_TC = 0, 1, 2
-TSID_CLIP_NONE, TSID_CLIP_ASYM_STEP, TSID_CLIP_ASYM_GRAD = 0, 1, 2
+TSID_CLIP_NONE, TSID_CLIP_ASYM_STEP, TSID_CLIP_ASYM_GRAD, TSID_CLIP_ASYM_ENTRY = 0, 1, 2, 3
 TSID_NORM_NONE, TSID_NORM_COUNT = 0, 1
 TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
 

@@ -23,10 +23,14 @@ tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
   if (c->nnz > 2147483647LL) { snprintf(err, 256, "nnz exceeds 2^31-1"); return TSID_ERR_UNSUPPORTED; }
   if (c->precision != TSID_F32 && c->precision != TSID_BF16_SHADOW) { snprintf(err, 256, "bad precision"); return TSID_ERR_INVALID_ARG; }
   if (c->path < TSID_PATH_AUTO || c->path > TSID_PATH_DENSE_TC) { snprintf(err, 256, "bad path"); return TSID_ERR_INVALID_ARG; }
-  if (c->clip < TSID_CLIP_NONE || c->clip > TSID_CLIP_ASYM_GRAD) { snprintf(err, 256, "bad clip mode"); return TSID_ERR_INVALID_ARG; }
+  if (c->clip < TSID_CLIP_NONE || c->clip > TSID_CLIP_ASYM_ENTRY) { snprintf(err, 256, "bad clip mode"); return TSID_ERR_INVALID_ARG; }
   if (c->norm_p < 0 || c->norm_p > 1 || c->norm_q < 0 || c->norm_q > 1) { snprintf(err, 256, "bad norm mode"); return TSID_ERR_INVALID_ARG; }
   const int mult = c->precision == TSID_BF16_SHADOW ? 8 : 4;
   if (c->k < 1 || c->k > 256 || c->k % mult) { snprintf(err, 256, "k must be in [1,256] and a multiple of %d", mult); return TSID_ERR_UNSUPPORTED; }
+  if (c->clip == TSID_CLIP_ASYM_ENTRY && (c->path == TSID_PATH_DENSE_TC || (c->precision == TSID_F32 && c->k > 128))) {
+    snprintf(err, 256, "entry-wise clipping runs on the sparse path only (fp32 factors: k <= 128)");
+    return TSID_ERR_UNSUPPORTED;
+  }
   if (c->clip != TSID_CLIP_NONE && !(c->xi > 0.f)) { snprintf(err, 256, "xi must be > 0 when clipping"); return TSID_ERR_INVALID_ARG; }
   return TSID_OK;
 }
@@ -35,7 +39,8 @@ tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
 // its cells are observed; the answer depends on cfg alone, so the workspace size is predictable.
 int resolve_path(const tsid_config_t &c) {
   if (c.path != TSID_PATH_AUTO) return c.path;
-  if (dense_qualifies(c) && (double)c.nnz >= 0.05 * (double)c.m * (double)c.n) return TSID_PATH_DENSE_TC;
+  if (dense_qualifies(c) && c.clip != TSID_CLIP_ASYM_ENTRY && (double)c.nnz >= 0.05 * (double)c.m * (double)c.n)
+    return TSID_PATH_DENSE_TC;
   return TSID_PATH_SPARSE;
 }
 

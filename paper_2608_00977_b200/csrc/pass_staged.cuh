@@ -41,6 +41,16 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// One entry's contribution to one coordinate of the gradient row.  Aggregated modes: e * y.  Entry-wise
+// clip (Sec. 5.3 applied to every observed entry): min(2 e y - 2 lambda x, xi), nothing for padding
+// lanes of a ragged chunk (for xi > 0 the nested min/max of the paper equals min(d, xi)).
+template <bool ENTRY>
+__device__ __forceinline__ float entry_acc(float e, float y, float x, float acc, float lam2, float xi, bool valid) {
+  if (!ENTRY) return fmaf(e, y, acc);
+  const float d = fmaf(-lam2, x, 2.f * e * y);
+  return valid ? acc + fminf(d, xi) : acc;
+}
+
 // Minimum resident CTAs asked of the compiler: for 256-byte bf16 rows a cap of 96 registers (18 CTAs
 // per SM) measured 9 % faster than the unconstrained 101; tighter caps spill and lose.
 template <int KP, bool BF16>
@@ -48,12 +58,12 @@ struct StagedMinBlocks {
   static constexpr int value = KP <= 64 ? 32 : (KP == 128 ? 18 : 1);
 };
 
-template <int KP, bool BF16, int NST, int ROWS>
+template <int KP, bool BF16, int NST, int ROWS, bool ENTRY>
 __global__ void __launch_bounds__(32, StagedMinBlocks<KP, BF16>::value)
 pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__restrict__ idx,
                    const float *__restrict__ val, const void *__restrict__ stage_v,
                    const void *__restrict__ gather_v, int k, float *__restrict__ G,
-                   float *__restrict__ partial) {
+                   float *__restrict__ partial, float lam2, float xi) {
   using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
   constexpr int GROUP = Geo<KP>::GROUP, EPL = Geo<KP>::EPL, EPW = Geo<KP>::EPW;
   constexpr int VE = BF16 ? (EPL >= 8 ? 8 : 4) : 4;
@@ -195,9 +205,9 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
             }
             const float ea = ra - da, eb = rb - db;
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, true);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, true);
           }
         } else {
           const int iters = (nv + EPW - 1) / EPW;
@@ -228,9 +238,9 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
             const float ea = va ? ra - da : 0.f;
             const float eb = vb ? rb - db : 0.f;
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(ea, fa[i], acc[i]);
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = fmaf(eb, fb[i], acc[i]);
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
           }
         }
         __syncwarp();  // every lane is done reading this stage before it is refilled
@@ -259,12 +269,13 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
   }
 }
 
-template <int KP, bool BF16, int NST, int ROWS>
+template <int KP, bool BF16, int NST, int ROWS, bool ENTRY>
 cudaError_t launch_staged_t(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
   using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
   constexpr int smem = NST * ROWS * KP * (int)sizeof(T);
-  auto kern = pass_staged_kernel<KP, BF16, NST, ROWS>;
+  auto kern = pass_staged_kernel<KP, BF16, NST, ROWS, ENTRY>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  kern<<<sd.nseg, 32, smem, t->stream>>>(sd.segs, sd.nseg, sd.idx, sd.val, stage, gather, t->cfg.k, G, t->partial);
+  kern<<<sd.nseg, 32, smem, t->stream>>>(sd.segs, sd.nseg, sd.idx, sd.val, stage, gather, t->cfg.k, G, t->partial,
+                                         2.0f * t->cfg.lambda, t->cfg.xi);
   return cudaGetLastError();
 }

@@ -222,7 +222,7 @@ __device__ __forceinline__ float clip_dir(float d, float xi, int clip) {
 
 // D = G * (2/s) - 2 lambda X; clip; X += eta D; refresh the bf16 shadow; flag non-finite values.
 __global__ void __launch_bounds__(256)
-update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int clip, int32_t *flags) {
+update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int clip, float gmul, int32_t *flags) {
   const int64_t total = a.n4 + b.n4;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   bool bad = false;
@@ -230,7 +230,7 @@ update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int
     const bool first = i < a.n4;
     const UpdSide &sd = first ? a : b;
     const int64_t j = first ? i : i - a.n4;
-    const float sc = __ldg(sd.scale + j / k4);
+    const float sc = __ldg(sd.scale + j / k4) * gmul;
     float4 x = reinterpret_cast<float4 *>(sd.X)[j];
     const float4 gv = __ldcs(reinterpret_cast<const float4 *>(sd.G) + j);
     float xs[4] = {x.x, x.y, x.z, x.w};
@@ -359,21 +359,27 @@ cudaError_t launch_pass_k(cudaStream_t st, const Side &sd, const void *stage, co
 // Chunk depth measured on B200: two stages; 16-row chunks for 256-byte rows and wider (more CTAs
 // per SM matter more than deeper chunks), 32-row chunks below.  Returns cudaErrorNotSupported when
 // there is no staged instantiation (fp32 with k > 128): the caller then uses the direct kernel.
-cudaError_t launch_staged(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+template <bool ENTRY>
+cudaError_t launch_staged_e(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
   if (sd.nseg <= 0) return cudaSuccess;
   const int k = t->cfg.k;
   if (t->cfg.precision == TSID_BF16_SHADOW) {
-    if (k <= 16) return launch_staged_t<16, true, 2, 32>(t, sd, stage, gather, G);
-    if (k <= 32) return launch_staged_t<32, true, 2, 32>(t, sd, stage, gather, G);
-    if (k <= 64) return launch_staged_t<64, true, 2, 32>(t, sd, stage, gather, G);
-    if (k <= 128) return launch_staged_t<128, true, 2, 16>(t, sd, stage, gather, G);
-    return launch_staged_t<256, true, 2, 16>(t, sd, stage, gather, G);
+    if (k <= 16) return launch_staged_t<16, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 32) return launch_staged_t<32, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 64) return launch_staged_t<64, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 128) return launch_staged_t<128, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
+    return launch_staged_t<256, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
   }
-  if (k <= 16) return launch_staged_t<16, false, 2, 32>(t, sd, stage, gather, G);
-  if (k <= 32) return launch_staged_t<32, false, 2, 32>(t, sd, stage, gather, G);
-  if (k <= 64) return launch_staged_t<64, false, 2, 16>(t, sd, stage, gather, G);
-  if (k <= 128) return launch_staged_t<128, false, 2, 16>(t, sd, stage, gather, G);
+  if (k <= 16) return launch_staged_t<16, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 32) return launch_staged_t<32, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 64) return launch_staged_t<64, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 128) return launch_staged_t<128, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
   return cudaErrorNotSupported;
+}
+
+cudaError_t launch_staged(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+  if (t->cfg.clip == TSID_CLIP_ASYM_ENTRY) return launch_staged_e<true>(t, sd, stage, gather, G);
+  return launch_staged_e<false>(t, sd, stage, gather, G);
 }
 
 template <int MODE>
@@ -435,7 +441,11 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
   UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4};
   UpdSide b{d_Q, GQ, t->colside.scale, t->colside.shadow, (int64_t)c.n * c.k / 4};
   prof_mark(t, EV_UPD0);
-  update_kernel<<<ew_grid(a.n4 + b.n4), 256, 0, t->stream>>>(a, b, c.k / 4, c.eta, 2.0f * c.lambda, c.xi, c.clip,
+  // entry-wise clip: the passes already delivered the sum of clipped per-entry directions (regulariser
+  // included), so the update is x += eta * G / s   (scale holds 2 / s)
+  const bool entry = c.clip == TSID_CLIP_ASYM_ENTRY;
+  update_kernel<<<ew_grid(a.n4 + b.n4), 256, 0, t->stream>>>(a, b, c.k / 4, c.eta, entry ? 0.f : 2.0f * c.lambda, c.xi,
+                                                             entry ? (int)TSID_CLIP_NONE : c.clip, entry ? 0.5f : 1.0f,
                                                              t->flags);
   prof_mark(t, EV_UPD1);
   if (t->prof.on && t->prof.nsteps < kProfSteps) t->prof.nsteps++;

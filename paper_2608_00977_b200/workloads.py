@@ -21,7 +21,7 @@ from dataclasses import dataclass, replace
 
 import torch
 
-CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD = 0, 1, 2
+CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD, CLIP_ASYM_ENTRY = 0, 1, 2, 3
 NORM_NONE, NORM_COUNT = 0, 1
 
 

@@ -47,7 +47,7 @@ def test_k_multiple_of_4_fp32():
         _assert_step(W.make_template(w, DEV, order="shuffled"), B.TSID_F32)
 
 
-@pytest.mark.parametrize("clip", [W.CLIP_NONE, W.CLIP_ASYM_STEP, W.CLIP_ASYM_GRAD])
+@pytest.mark.parametrize("clip", [W.CLIP_NONE, W.CLIP_ASYM_STEP, W.CLIP_ASYM_GRAD, W.CLIP_ASYM_ENTRY])
 @pytest.mark.parametrize("norm_p,norm_q", [(0, 0), (0, 1), (1, 1)])
 def test_modes(clip, norm_p, norm_q):
     w = small_workload("modes", 900, 1300, 32, 60_000, positions="zipf", seed=5, values="ratings", noise_var=0.25,
@@ -59,6 +59,19 @@ def test_modes(clip, norm_p, norm_q):
         inc = P1 - tpl.P0.cpu().numpy()
         assert inc.max() <= w.eta * w.xi * (1 + 1e-5) and np.isclose(inc.max(), w.eta * w.xi, rtol=1e-5)
         assert inc.min() < -w.eta * w.xi
+
+
+@pytest.mark.parametrize("precision", [B.TSID_F32, B.TSID_BF16_SHADOW])
+@pytest.mark.parametrize("k", [16, 40, 64, 128])
+def test_entrywise_clip_rank_sweep(k, precision):
+    """Sec. 5.3 applied entry by entry (literal Eq. 9 normalisation: q side only), every staged instantiation."""
+    w = small_workload("entry-k%d" % k, 1200, 900, k, 70_000 + 7, positions="zipf", seed=300 + k, values="ratings",
+                       noise_var=0.25, eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_ENTRY, norm_p=W.NORM_NONE,
+                       norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    _assert_step(tpl, precision)
+    T, P1, _, GP, _ = gpu_step(tpl, precision=precision)
+    assert GP.max() <= 0.1 * np.bincount(tpl.rows.cpu().numpy(), minlength=w.m).max() + 1e-3   # each term <= xi
 
 
 def test_split_rows_and_empty_rows():
