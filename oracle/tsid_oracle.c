@@ -340,3 +340,64 @@ void orc_sample_template(int32_t m, int32_t n, int64_t nnz, double alpha, uint64
   *nnz_out = o;
   free(ck);
 }
+
+/* ---- Stage II: template-conditioned extension (Sec. 5.2, Eq. 10) ---------------------------------
+ * With the template estimate Rhat* = P Q^T (m x d) fixed, every column j of the full matrix gets a
+ * coefficient vector C_j in R^d minimising
+ *       L_j(C_j) = sum_{i in Omega^j} (R_ij - Rhat*_i C_j)^2 + lambda |C_j|^2        (Eq. 10, per column)
+ * by gradient steps through Adam (Kingma & Ba, Algorithm 1):
+ *       g = -2 Rhat*_{Omega^j}^T e + 2 lambda C_j,     e_i = R_ij - Rhat*_i C_j
+ *       m <- b1 m + (1-b1) g,  v <- b2 v + (1-b2) g^2,  C_j <- C_j - eta (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + eps)
+ * Readings: C starts at the values passed in (zeros in the tests and the bench); Adam's constants are
+ * arguments (the paper names the optimiser only); the objective decomposes over columns, so a chunk is
+ * just a set of columns and chunking cannot change the result; `iters` steps per column.
+ * The loops below follow the definition with Rhat* materialised (no factored shortcut).
+ * Layout: column-compressed input (col_ptr[ncols+1], row_idx, vals); C is stored one column after the
+ * other, C[j*d + a].  sse_out (may be NULL) receives sum_Omega e^2 at the returned C. */
+void orc_extend(int32_t m, int32_t d, int32_t k, int32_t ncols, const int64_t *col_ptr,
+                const int32_t *row_idx, const float *vals, const float *P, const float *Q,
+                double eta, double lambda, double b1, double b2, double eps, int32_t iters,
+                double *C, double *sse_out) {
+  double *Rhat = (double *)malloc(sizeof(double) * (size_t)m * d);
+  for (int32_t i = 0; i < m; ++i)
+    for (int32_t a = 0; a < d; ++a) {
+      double s = 0.0;
+      for (int32_t l = 0; l < k; ++l) s += (double)P[(size_t)i * k + l] * (double)Q[(size_t)a * k + l];
+      Rhat[(size_t)i * d + a] = s;
+    }
+  double *g = (double *)malloc(sizeof(double) * (size_t)d);
+  double *mo = (double *)malloc(sizeof(double) * (size_t)d);
+  double *vo = (double *)malloc(sizeof(double) * (size_t)d);
+  double sse = 0.0;
+  for (int32_t j = 0; j < ncols; ++j) {
+    double *Cj = C + (size_t)j * d;
+    for (int32_t a = 0; a < d; ++a) { mo[a] = 0.0; vo[a] = 0.0; }
+    double p1 = 1.0, p2 = 1.0;
+    for (int32_t it = 1; it <= iters; ++it) {
+      for (int32_t a = 0; a < d; ++a) g[a] = 2.0 * lambda * Cj[a];
+      for (int64_t t = col_ptr[j]; t < col_ptr[j + 1]; ++t) {
+        const double *rh = Rhat + (size_t)row_idx[t] * d;
+        double pred = 0.0;
+        for (int32_t a = 0; a < d; ++a) pred += rh[a] * Cj[a];
+        double e = (double)vals[t] - pred;
+        for (int32_t a = 0; a < d; ++a) g[a] -= 2.0 * e * rh[a];
+      }
+      p1 *= b1; p2 *= b2;
+      for (int32_t a = 0; a < d; ++a) {
+        mo[a] = b1 * mo[a] + (1.0 - b1) * g[a];
+        vo[a] = b2 * vo[a] + (1.0 - b2) * g[a] * g[a];
+        double mh = mo[a] / (1.0 - p1), vh = vo[a] / (1.0 - p2);
+        Cj[a] -= eta * mh / (sqrt(vh) + eps);
+      }
+    }
+    for (int64_t t = col_ptr[j]; t < col_ptr[j + 1]; ++t) {
+      const double *rh = Rhat + (size_t)row_idx[t] * d;
+      double pred = 0.0;
+      for (int32_t a = 0; a < d; ++a) pred += rh[a] * Cj[a];
+      double e = (double)vals[t] - pred;
+      sse += e * e;
+    }
+  }
+  if (sse_out) *sse_out = sse;
+  free(Rhat); free(g); free(mo); free(vo);
+}
