@@ -224,6 +224,49 @@ def measure_sampling(args, w, tpl, B, dev):
                                    "frac": alg / (ms * 1e-3) / 1e9 / peak, "alg_bytes": alg}}))
 
 
+def measure_extend(args, w, tpl, B, dev):
+    """Times tsid_extend: the workload's matrix (all n columns, host-resident, column-compressed) is extended
+    from a template of d = n/4 columns (random-init factors of the workload's rank), `iters` Adam steps per
+    chunk, 16 chunks.  The timed region is the whole call: H2D of the entries, compute, D2H of C."""
+    d = max(8, w.n // 4)
+    iters = 10
+    chunk = max(1, (w.n + 15) // 16)
+    order = torch.argsort(tpl.cols.long() * w.m + tpl.rows.long())
+    rows = tpl.rows[order].cpu().pin_memory()
+    vals = tpl.vals[order].cpu().pin_memory()
+    counts = torch.bincount(tpl.cols.long(), minlength=w.n)
+    col_ptr = torch.zeros(w.n + 1, dtype=torch.int64)
+    col_ptr[1:] = torch.cumsum(counts.cpu(), 0)
+    col_ptr = col_ptr.pin_memory()
+    P = tpl.P0
+    Q = tpl.Q0[:d].contiguous()
+    Ch = torch.zeros(w.n, d).pin_memory()
+    times = []
+    for it in range(args.warmup + args.steps):
+        Ch.zero_()
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        B.tsid_extend(P, Q, col_ptr, rows, vals, Ch, chunk, iters, 0.02, 0.05, cold_start=True)
+        torch.cuda.synchronize(dev)
+        if it >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    t = sum(times) / len(times)
+    nnz = tpl.nnz
+    # per Adam step: C, m, v read + written (24 B per coefficient) + C read by the first GEMM (4 B)
+    # + the entry pass (8 + 4k B per entry, fp32 gathers); per call: entries in (8 B) and C in/out (8 B)
+    alg_dev = iters * (w.n * d * 28 + nnz * (8 + 4 * w.k))
+    flops = iters * (4.0 * w.n * d * w.k + 4.0 * nnz * w.k)
+    peak = load_peaks()[0]
+    print(json.dumps({"metric": "Stage II observed-entry Adam updates/sec", "value": nnz * iters / t, "unit": "updates/s",
+                      "s_per_call": t, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "config": {"workload": w.name, "m": w.m, "n_cols": w.n, "d": d, "k": w.k, "nnz": nnz,
+                                 "iters": iters, "chunk_cols": chunk, "dtype": "f32"},
+                      "h2d_bytes_per_call": nnz * 8 + (w.n + 1) * 8, "d2h_bytes_per_call": w.n * d * 4,
+                      "roofline": {"bound": "hbm", "achieved": alg_dev / t / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": alg_dev / t / 1e9 / peak, "alg_bytes": alg_dev,
+                                   "fp32_tflops": flops / t / 1e12}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -233,8 +276,9 @@ def main():
     ap.add_argument("--impl", default="tsid")
     ap.add_argument("--path", default="sparse", choices=["auto", "sparse", "dense"],
                     help="kernel path of the measured template (the dense tcgen05 variant needs a qualifying workload, e.g. C4)")
-    ap.add_argument("--measure", default="step", choices=["step", "sample"],
-                    help="step: the gradient step (default); sample: tsid_sample_template on the workload's COO")
+    ap.add_argument("--measure", default="step", choices=["step", "sample", "extend"],
+                    help="step: the gradient step (default); sample: tsid_sample_template on the workload's COO; "
+                         "extend: Stage II (tsid_extend) of the workload's matrix on a template of a quarter of its columns")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -273,6 +317,9 @@ def main():
     nnz = tpl.nnz
     if args.measure == "sample":
         measure_sampling(args, w, tpl, B, dev)
+        return
+    if args.measure == "extend":
+        measure_extend(args, w, tpl, B, dev)
         return
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
     want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]

@@ -207,6 +207,42 @@ tsid_status_t tsid_sample_template(int32_t m, int32_t n, int64_t nnz, double alp
                                    int32_t *d_colmap, int32_t *d_rows_out, int32_t *d_cols_out,
                                    float *d_vals_out, int32_t *h_d_out, int64_t *h_nnz_out);
 
+/* Stage II, the template-conditioned extension (Sec. 5.2, Eq. 10).  With the template estimate
+ * Rhat* = P Q^T (m x d) fixed, every column j of the matrix being completed gets coefficients C_j in R^d
+ * minimising  sum_{i in Omega^j} (R_ij - Rhat*_i C_j)^2 + lambda |C_j|^2  by `iters` Adam steps
+ * (Kingma & Ba, Algorithm 1, bias-corrected; beta1, beta2, eps as given).  Columns are processed in
+ * chunks of `chunk_cols`: the matrix and C stay in HOST memory (pinned memory makes the copies
+ * asynchronous), the template factors stay on the device, and while one chunk computes the next one is
+ * copied in and the previous one's coefficients are copied out.
+ *   - d_P (m x k), d_Q (d x k): DEVICE, fp32 row-major, the fitted template factors; only read.
+ *   - h_col_ptr (int64[n_cols + 1]), h_row_idx (int32[nnz]), h_vals (fp32[nnz]): HOST, the observed
+ *     entries in column-compressed order (entries of column j at positions [col_ptr[j], col_ptr[j+1])).
+ *   - h_C: HOST, fp32 [n_cols x d], column j's coefficients at h_C + j*d; read as the starting point
+ *     (zeros for a cold start) and overwritten with the result.
+ *   - h_sse_or_null: HOST, receives sum_Omega e^2 at the returned coefficients.
+ *   - cfg.workspace: DEVICE, tsid_extend_workspace_bytes(cfg, h_col_ptr) bytes (it depends on the
+ *     largest chunk); nothing is allocated on the device.  The call creates two helper streams and a
+ *     few events, and synchronises before it returns.
+ * Limits: k a multiple of 4 in [4, 128]; at most 2^31 - 3 entries per chunk.  Errors: INVALID_ARG,
+ * UNSUPPORTED (k), OOM (workspace), INDEX_RANGE (a row index outside [0, m)), CUDA. */
+enum { TSID_EXTEND_COLD_START = 1u };
+typedef struct {
+  int32_t m, d, k;     /* rows; template columns (rows of Q); rank                      */
+  int32_t n_cols;      /* columns handled by this call                                  */
+  int32_t chunk_cols;  /* chunk width (Delta c)                                         */
+  int32_t iters;       /* Adam steps per chunk                                          */
+  float eta, lambda, beta1, beta2, eps;
+  uint32_t flags;      /* TSID_EXTEND_COLD_START: start from C = 0, h_C is only written */
+  void *stream;           /* compute stream (cudaStream_t) owned by the caller          */
+  void *workspace;        /* DEVICE memory owned by the caller, 256-byte aligned        */
+  size_t workspace_bytes;
+} tsid_extend_config_t;
+tsid_status_t tsid_extend_workspace_bytes(const tsid_extend_config_t *cfg, const int64_t *h_col_ptr,
+                                          size_t *h_bytes_out);
+tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, const float *d_Q,
+                          const int64_t *h_col_ptr, const int32_t *h_row_idx, const float *h_vals,
+                          float *h_C, double *h_sse_or_null);
+
 /* Per-kernel timing for benchmarks.  tsid_set_profiling(t, 1) makes every following step record
  * CUDA events on the template's stream right before and after its row pass, its column pass
  * and its update kernel (at most 256 steps are kept); 0 turns it off and frees the events.

@@ -31,7 +31,8 @@ TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
 EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",
            "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
-           "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template"]
+           "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
+           "tsid_extend_workspace_bytes", "tsid_extend"]
 
 
 class TsidConfig(C.Structure):
@@ -41,6 +42,13 @@ class TsidConfig(C.Structure):
                 ("clip", C.c_int32), ("norm_p", C.c_int32), ("norm_q", C.c_int32),
                 ("flags", C.c_uint32), ("stream", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t)]
+
+
+class TsidExtendConfig(C.Structure):
+    _fields_ = [("m", C.c_int32), ("d", C.c_int32), ("k", C.c_int32), ("n_cols", C.c_int32),
+                ("chunk_cols", C.c_int32), ("iters", C.c_int32),
+                ("eta", C.c_float), ("lam", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("flags", C.c_uint32), ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
 class TsidError(RuntimeError):
@@ -81,6 +89,8 @@ def lib():
         L.tsid_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
         L.tsid_sample_template.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_uint64, vp, vp, vp, vp, vp,
                                            C.c_size_t, vp, vp, vp, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+        L.tsid_extend_workspace_bytes.argtypes = [C.POINTER(TsidExtendConfig), vp, C.POINTER(C.c_size_t)]
+        L.tsid_extend.argtypes = [C.POINTER(TsidExtendConfig), vp, vp, vp, vp, vp, vp, C.POINTER(C.c_double)]
         L.tsid_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name != "tsid_last_error":
@@ -321,6 +331,44 @@ def tsid_sample_template(m, n, rows, cols, vals, alpha, seed, stream=None):
         raise TsidError(st, "tsid_sample_template")
     k = kept.value
     return colmap, ro[:k], co[:k], vo[:k], d.value
+
+
+TSID_EXTEND_COLD_START = 1
+
+
+def tsid_extend(P, Q, col_ptr, row_idx, vals, C0, chunk_cols, iters, eta, lam, beta1=0.9, beta2=0.999, eps=1e-8,
+                want_sse=False, stream=None, cold_start=False):
+    """Stage II extension.  P (m x k), Q (d x k): CUDA fp32 tensors.  col_ptr (int64), row_idx (int32),
+    vals (fp32), C0 (fp32 [n_cols, d]): CPU tensors (pinned for asynchronous copies); C0 is overwritten with
+    the fitted coefficients.  Returns the SSE if requested."""
+    m, k = P.shape
+    d = Q.shape[0]
+    n_cols = col_ptr.numel() - 1
+    for t, dt in ((col_ptr, torch.int64), (row_idx, torch.int32), (vals, torch.float32), (C0, torch.float32)):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors of the documented dtypes")
+    _check_tensor(P, torch.float32, m * k, "P")
+    _check_tensor(Q, torch.float32, d * k, "Q")
+    if C0.numel() != n_cols * d:
+        raise ValueError("C0 must have n_cols * d elements")
+    dev = P.device
+    stream = stream if stream is not None else torch.cuda.current_stream(dev)
+    cfg = TsidExtendConfig(m, d, k, n_cols, chunk_cols, iters, eta, lam, beta1, beta2, eps,
+                           TSID_EXTEND_COLD_START if cold_start else 0, stream.cuda_stream, None, 0)
+    need = C.c_size_t(0)
+    st = lib().tsid_extend_workspace_bytes(C.byref(cfg), col_ptr.data_ptr(), C.byref(need))
+    if st != TSID_OK:
+        raise TsidError(st, "tsid_extend_workspace_bytes")
+    ws = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    cfg.workspace = (ws.data_ptr() + 255) & ~255
+    cfg.workspace_bytes = need.value
+    sse = C.c_double(0)
+    with torch.cuda.device(dev):
+        st = lib().tsid_extend(C.byref(cfg), P.data_ptr(), Q.data_ptr(), col_ptr.data_ptr(), row_idx.data_ptr(),
+                               vals.data_ptr(), C0.data_ptr(), C.byref(sse) if want_sse else None)
+    if st != TSID_OK:
+        raise TsidError(st, "tsid_extend")
+    return sse.value if want_sse else None
 
 
 def template_from_workload(tpl, path=TSID_PATH_AUTO, flags=0, precision=None) -> Template:

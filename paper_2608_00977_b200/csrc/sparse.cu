@@ -331,6 +331,13 @@ __global__ void __launch_bounds__(256) reduce_final_kernel(const double *__restr
   if (threadIdx.x == 0) { out2[0] = va; out2[1] = vb; }
 }
 
+// *out += sum a[0..RED_BLOCKS)
+__global__ void __launch_bounds__(256) reduce_add_kernel(const double *__restrict__ a, double *__restrict__ out) {
+  double v = threadIdx.x < RED_BLOCKS ? a[threadIdx.x] : 0.0;
+  v = block_sum(v);
+  if (threadIdx.x == 0) *out += v;
+}
+
 // ---- dispatch -------------------------------------------------------------------------------------------
 template <int KP, bool BF16, int MODE>
 cudaError_t launch_pass_t(cudaStream_t st, const Side &sd, const void *stage, const void *gather, int k,
@@ -473,6 +480,24 @@ cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, do
   sqnorm_slices_kernel<<<RED_BLOCKS, 256, 0, t->stream>>>(d_P, (int64_t)t->cfg.m * t->cfg.k, d_Q,
                                                          (int64_t)t->cfg.n * t->cfg.k, sl_b);
   reduce_final_kernel<<<1, 256, 0, t->stream>>>(sl_a, sl_b, d_out2);
+  return cudaGetLastError();
+}
+
+// One side's gather-reduce pass on its own (used by the Stage II extension): G[row] = sum over the
+// row's entries of e * gathered row, e = val - staged row . gathered row; fp32 or bf16 per t->cfg.
+cudaError_t sparse_side_grad(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+  CK(launch_pass<MODE_GRAD>(t, sd, stage, gather, G, nullptr, nullptr));
+  if (sd.nsplit > 0) fixup_kernel<<<sd.nsplit, 128, 0, t->stream>>>(sd.splits, sd.nsplit, t->partial, G, t->cfg.k);
+  return cudaGetLastError();
+}
+
+// d_out[0] += sum over the side's entries of e^2 (fixed order inside; `red` needs 2 + 2*256 + nseg doubles)
+cudaError_t sparse_side_sse(tsid_template *t, const Side &sd, const void *stage, const void *gather, double *red,
+                            double *d_out) {
+  double *warp_part = red + 2 + 2 * RED_BLOCKS, *sl_a = red + 2;
+  CK(launch_pass<MODE_LOSS>(t, sd, stage, gather, nullptr, nullptr, warp_part));
+  reduce_slices_kernel<<<RED_BLOCKS, 256, 0, t->stream>>>(warp_part, sd.nseg, sl_a);
+  reduce_add_kernel<<<1, 256, 0, t->stream>>>(sl_a, d_out);
   return cudaGetLastError();
 }
 

@@ -1,0 +1,84 @@
+"""Stage II extension (Sec. 5.2, Eq. 10 + Adam): CUDA path against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import relerr
+from paper_2608_00977_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _problem(m, d, k, ncols, per_col, seed, hot=None):
+    rng = np.random.default_rng(seed)
+    P = (rng.standard_normal((m, k)) * k ** -0.25).astype(np.float32)
+    Q = (rng.standard_normal((d, k)) * k ** -0.25).astype(np.float32)
+    cols = []
+    for j in range(ncols):
+        cnt = per_col if hot is None or j not in hot else hot[j]
+        cnt = min(m, int(rng.integers(max(0, cnt - cnt // 2), cnt + cnt // 2 + 1)))
+        cols.append(np.sort(rng.choice(m, cnt, replace=False)))
+    cols[min(3, ncols - 1)] = cols[0][:0]                      # one column without observations
+    col_ptr = np.concatenate([[0], np.cumsum([len(c) for c in cols])]).astype(np.int64)
+    row_idx = np.concatenate(cols).astype(np.int32)
+    vals = (rng.standard_normal(len(row_idx)) * 1.5).astype(np.float32)
+    return P, Q, col_ptr, row_idx, vals
+
+
+def _run_gpu(P, Q, cp, ri, v, chunk, iters, eta, lam, C0=None):
+    ncols, d = len(cp) - 1, Q.shape[0]
+    Ch = torch.zeros(ncols, d) if C0 is None else torch.tensor(C0, dtype=torch.float32)
+    Ch = Ch.pin_memory()
+    sse = B.tsid_extend(torch.tensor(P, device=DEV), torch.tensor(Q, device=DEV), torch.tensor(cp).pin_memory(),
+                        torch.tensor(ri).pin_memory(), torch.tensor(v).pin_memory(), Ch, chunk, iters, eta, lam,
+                        want_sse=True)
+    return Ch.numpy().copy(), sse
+
+
+@pytest.mark.parametrize("m,d,k,ncols,per_col,chunk", [(500, 96, 32, 300, 60, 64), (300, 40, 16, 130, 30, 1000),
+                                                       (800, 200, 64, 257, 80, 100), (64, 8, 4, 5, 10, 2)])
+def test_extend_matches_oracle(m, d, k, ncols, per_col, chunk):
+    P, Q, cp, ri, v = _problem(m, d, k, ncols, per_col, seed=m + d)
+    eta, lam, iters = 0.02, 0.05, 15
+    C, sse = _run_gpu(P, Q, cp, ri, v, chunk, iters, eta, lam)
+    Cr, sse_r = oracle.extend(m, d, k, cp, ri, v, P, Q, eta, lam, iters)
+    assert relerr(C, Cr) <= 2e-3, relerr(C, Cr)     # Adam divides by sqrt(v): fp32 noise on tiny gradients is amplified
+    assert abs(sse - sse_r) / sse_r <= 1e-3
+    assert not C[min(3, ncols - 1)].any()
+
+
+def test_extend_chunking_is_invisible_and_loss_decreases():
+    P, Q, cp, ri, v = _problem(1200, 64, 32, 400, 2500 // 8, seed=9, hot={7: 1200, 100: 1100})   # split columns
+    outs = [_run_gpu(P, Q, cp, ri, v, chunk, 10, 0.02, 0.05) for chunk in (400, 64, 7)]
+    for C, sse in outs[1:]:
+        assert np.array_equal(C, outs[0][0])             # bitwise: columns are independent
+        assert abs(sse - outs[0][1]) <= 1e-12 * sse      # chunk totals are added in a different order
+    sse0 = float(np.sum(v.astype(np.float64) ** 2))                            # C = 0 predicts 0
+    assert outs[0][1] < 0.95 * sse0
+    # warm start: 6 + 4 steps is not the same as 10 (Adam's moments restart), but it keeps descending
+    C6, s6 = _run_gpu(P, Q, cp, ri, v, 64, 6, 0.02, 0.05)
+    C10, s10 = _run_gpu(P, Q, cp, ri, v, 64, 4, 0.02, 0.05, C0=C6)
+    assert s10 < s6
+
+
+def test_extend_cold_start_ignores_host_contents():
+    P, Q, cp, ri, v = _problem(300, 40, 16, 130, 30, seed=4)
+    ref, _ = _run_gpu(P, Q, cp, ri, v, 50, 8, 0.02, 0.05)
+    Ch = torch.full((130, 40), 7.0).pin_memory()
+    B.tsid_extend(torch.tensor(P, device=DEV), torch.tensor(Q, device=DEV), torch.tensor(cp).pin_memory(),
+                  torch.tensor(ri).pin_memory(), torch.tensor(v).pin_memory(), Ch, 50, 8, 0.02, 0.05, cold_start=True)
+    assert np.array_equal(Ch.numpy(), ref)
+
+
+def test_extend_errors():
+    P, Q, cp, ri, v = _problem(64, 8, 4, 5, 10, seed=1)
+    bad = ri.copy(); bad[3] = 64
+    with pytest.raises(B.TsidError) as e:
+        _run_gpu(P, Q, cp, bad, v, 2, 3, 0.02, 0.05)
+    assert e.value.status == B.TSID_ERR_INDEX_RANGE
+    cfg = B.TsidExtendConfig(64, 8, 6, 5, 2, 3, 0.02, 0.05, 0.9, 0.999, 1e-8, 0, None, None, 0)
+    import ctypes as C
+    need = C.c_size_t(0)
+    assert B.lib().tsid_extend_workspace_bytes(C.byref(cfg), torch.tensor(cp).data_ptr(), C.byref(need)) == B.TSID_ERR_UNSUPPORTED
