@@ -113,7 +113,10 @@ def aggregate_value(world, units_per_rank_step, steps, seconds):
 
 
 def alg_bytes(w, nnz, nseg_row, nseg_col):
-    """Algorithmic bytes of one launch of each kernel of a step ("Roofline")."""
+    """Algorithmic bytes of one launch of each kernel of a step.  A pass reads per entry a 4-byte index, a
+    4-byte value and one gathered factor row (k*b bytes, b = 2 for bf16 shadows, 4 for fp32), and per row the
+    staged factor row (k*b), a 16-byte segment descriptor, and writes the gradient row (4k).  The update reads
+    gradient and master, writes master (and the bf16 shadow), and reads one scale per row."""
     b = 2 if w.precision == "bf16" else 4
     k = w.k
     row = nnz * (8 + k * b) + w.m * k * (b + 4) + nseg_row * 16

@@ -16,7 +16,7 @@
  *   - aggregated update and the 1/n normalisation: Sec. 5.1, Eq. 9
  *   - asymmetric clipping min(max(xi, -g), g): Sec. 5.3 (unnumbered equation)
  *
- * Readings taken where the paper is ambiguous (all listed in the design notes):
+ * Readings taken where the paper is ambiguous:
  *   - the symbol added to the factors in Eq. 9 is the step DIRECTION
  *       D = -grad L = 2 G / s - 2 lambda x,   G_P = E Q,  G_Q = E^T P,
  *     E the sparse residual matrix; the update is x + eta * D;
