@@ -227,6 +227,54 @@ def measure_sampling(args, w, tpl, B, dev):
                                    "frac": alg / (ms * 1e-3) / 1e9 / peak, "alg_bytes": alg}}))
 
 
+def measure_layout(args, w, tpl, B, dev):
+    """Times the layout pass (tsid_template_create on the sparse path: COO -> CSR, CSC, perm, pointers,
+    segments) of the workload's entries in the order `--order` gives them, workspace already allocated."""
+    import ctypes as C
+    nnz = tpl.nnz
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    cfg = B.make_config(w.m, w.n, w.k, nnz, prec, B.TSID_PATH_SPARSE, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q, 0)
+    need = C.c_size_t(0)
+    assert B.lib().tsid_workspace_bytes(C.byref(cfg), C.byref(need)) == B.TSID_OK
+    ws = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    cfg.workspace = (ws.data_ptr() + 255) & ~255
+    cfg.workspace_bytes = need.value
+    stream = torch.cuda.current_stream(dev)
+    cfg.stream = stream.cuda_stream
+    times = []
+    for it in range(args.warmup + args.steps):
+        h = C.c_void_p()
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        st = B.lib().tsid_template_create(C.byref(cfg), tpl.rows.data_ptr(), tpl.cols.data_ptr(), tpl.vals.data_ptr(),
+                                          C.byref(h))
+        torch.cuda.synchronize(dev)
+        dt = time.perf_counter() - t0
+        assert st == B.TSID_OK, st
+        B.lib().tsid_destroy(h)
+        if it >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    peak = load_peaks()[0]
+    # compulsory: the COO triples in (12 B), col_idx + val_csr out (8 B), row_idx + val_csc + perm out (12 B) per
+    # entry.  The radix passes of the implemented algorithm move more: per entry and pass 4 B (histogram) + the
+    # key and its payload words in and out; the third sort starts from the identity, so its first pass reads 12 B
+    # and writes 16 B.  Input check 8 B, the two pointer builds 8 B.
+    compulsory = nnz * 32 + (w.m + w.n + 2) * 8
+    pc = max(1, (max(w.n - 1, 1).bit_length() + 7) // 8)
+    pr = max(1, (max(w.m - 1, 1).bit_length() + 7) // 8)
+    third = pc * 4 + 28 + (pc - 1) * 32
+    per_entry = 16 + third + ((pc + pr) * 28 if args.order == "shuffled" else 16)
+    alg = nnz * per_entry
+    print(json.dumps({"metric": "entries laid out/sec", "value": nnz / t, "unit": "entries/s", "ms_per_call": t * 1e3,
+                      "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "config": {"workload": w.name, "order": args.order, "m": w.m, "n": w.n, "nnz": nnz,
+                                 "workspace_gb": need.value / 1e9},
+                      "roofline": {"bound": "hbm", "achieved": alg / t / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": alg / t / 1e9 / peak, "alg_bytes": alg, "alg_bytes_per_entry": per_entry,
+                                   "compulsory_bytes": compulsory, "compulsory_frac": compulsory / t / 1e9 / peak}}))
+
+
 def measure_extend(args, w, tpl, B, dev):
     """Times tsid_extend: the workload's matrix (all n columns, host-resident, column-compressed) is extended
     from a template of d = n/4 columns (random-init factors of the workload's rank), `iters` Adam steps per
@@ -279,9 +327,12 @@ def main():
     ap.add_argument("--impl", default="tsid")
     ap.add_argument("--path", default="sparse", choices=["auto", "sparse", "dense"],
                     help="kernel path of the measured template (the dense tcgen05 variant needs a qualifying workload, e.g. C4)")
-    ap.add_argument("--measure", default="step", choices=["step", "sample", "extend"],
+    ap.add_argument("--measure", default="step", choices=["step", "sample", "extend", "layout"],
                     help="step: the gradient step (default); sample: tsid_sample_template on the workload's COO; "
-                         "extend: Stage II (tsid_extend) of the workload's matrix on a template of a quarter of its columns")
+                         "extend: Stage II (tsid_extend) of the workload's matrix on a template of a quarter of its columns; "
+                         "layout: the layout pass (tsid_template_create) on the workload's COO in --order")
+    ap.add_argument("--order", default="shuffled", choices=["sorted", "shuffled"],
+                    help="entry order of the COO input for --measure layout")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -314,7 +365,7 @@ def main():
 
     w = W.CONFIGS[args.workload]
     t0 = time.perf_counter()
-    tpl = W.make_template(w, dev, order="sorted")
+    tpl = W.make_template(w, dev, order=args.order if args.measure == "layout" else "sorted")
     torch.cuda.synchronize(dev)
     t1 = time.perf_counter()
     nnz = tpl.nnz
@@ -323,6 +374,9 @@ def main():
         return
     if args.measure == "extend":
         measure_extend(args, w, tpl, B, dev)
+        return
+    if args.measure == "layout":
+        measure_layout(args, w, tpl, B, dev)
         return
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
     want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]

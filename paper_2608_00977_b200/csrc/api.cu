@@ -79,6 +79,8 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
   // transient buffers of the layout pass
   ls.kA = cv.take<uint32_t>(nz); ls.kB = cv.take<uint32_t>(nz);
   ls.vA = cv.take<uint32_t>(nz); ls.vB = cv.take<uint32_t>(nz);
+  ls.wA = cv.take<uint32_t>(nz); ls.wB = cv.take<uint32_t>(nz);
+  ls.xA = cv.take<uint32_t>(nz); ls.xB = cv.take<uint32_t>(nz);
   ls.hist = cv.take<uint32_t>(256 * (size_t)kSortBlocksMax);
   const size_t mx = (m > n ? m : n) + 2;
   ls.scanA = cv.take<uint32_t>(mx); ls.scanB = cv.take<uint32_t>(mx); ls.scanC = cv.take<uint32_t>(mx);

@@ -183,7 +183,7 @@ ExtCarve carve(void *base, const tsid_extend_config_t &c, int64_t cap) {
   e.red = cv.take<double>(2 + 2 * 256 + (size_t)e.cap_seg);
   e.sse = cv.take<double>(1);
   e.flags = cv.take<int32_t>(FLAG_COUNT);
-  e.ls.kA = e.ls.kB = e.ls.vA = e.ls.vB = nullptr;
+  e.ls.kA = e.ls.kB = e.ls.vA = e.ls.vB = e.ls.wA = e.ls.wB = e.ls.xA = e.ls.xB = nullptr;
   e.ls.hist = nullptr;
   e.ls.scanA = cv.take<uint32_t>(cc + 2);
   e.ls.scanB = cv.take<uint32_t>(cc + 2);

@@ -2,22 +2,26 @@
 // equal-length work segments of the two gather-reduce passes.  Integer work only; every
 // output is unique (stable sorts), so it can be compared bit for bit with a CPU sort.
 //
-// The sort is a hand-written stable LSD radix sort of (uint32 key, uint32 payload) pairs:
-// per pass a per-block digit histogram, an exclusive scan over the (digit, block) matrix and
-// a scatter that ranks the items of each tile in input order (warp match + per-warp digit
-// counters).  Integer atomics appear only in shared-memory histograms; nothing here
-// depends on their order.
+// The sort is a hand-written stable LSD radix sort of a uint32 key with one to three uint32
+// payload words: per pass a per-block digit histogram, an exclusive scan over the
+// (digit, block) matrix and a scatter that ranks the items of each tile in input order (warp
+// match + per-warp digit counters) and writes them out digit by digit from shared memory.
+// The index and the value of an entry travel with its key, so no pass gathers through a
+// permutation.  Integer atomics appear only in shared-memory histograms; nothing here depends
+// on their order.
 #include "tsid_internal.cuh"
 
 namespace tsid {
 
 namespace {
 
-constexpr int RS_THREADS = 256;
+constexpr int RS_HIST_THREADS = 256;
+constexpr int RS_THREADS = 512;  // scatter kernel
 constexpr int RS_WARPS = RS_THREADS / 32;
 constexpr int RS_ITEMS = 8;
-constexpr int RS_TILE = RS_THREADS * RS_ITEMS;  // 2048 pairs per tile
+constexpr int RS_TILE = RS_THREADS * RS_ITEMS;  // 4096 items per tile
 constexpr int RS_RADIX = 256;
+constexpr int RS_MAXP = 3;  // payload words carried per key
 
 #define CK(x)                        \
   do {                               \
@@ -26,31 +30,37 @@ constexpr int RS_RADIX = 256;
   } while (0)
 
 // ---- radix sort ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(RS_THREADS)
+// hist[d * nb + b] = number of keys of block b's range whose digit is d, for d <= mask.
+__global__ void __launch_bounds__(RS_HIST_THREADS)
 rs_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int64_t per_block, int shift,
                uint32_t mask, uint32_t *__restrict__ hist, int nb) {
   __shared__ uint32_t h[RS_RADIX];
-  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) h[d] = 0;
+  for (int d = threadIdx.x; d < RS_RADIX; d += RS_HIST_THREADS) h[d] = 0;
   __syncthreads();
   int64_t lo = (int64_t)blockIdx.x * per_block;
   int64_t hi = lo + per_block < n ? lo + per_block : n;
-  for (int64_t p = lo + threadIdx.x; p < hi; p += RS_THREADS)
+  for (int64_t p = lo + threadIdx.x; p < hi; p += RS_HIST_THREADS)
     atomicAdd(&h[(keys[p] >> shift) & mask], 1u);
   __syncthreads();
-  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) hist[(size_t)d * nb + blockIdx.x] = h[d];
+  for (int d = threadIdx.x; d <= (int)mask; d += RS_HIST_THREADS) hist[(size_t)d * nb + blockIdx.x] = h[d];
 }
 
-// Exclusive scan of a short array (<= 256 * kSortBlocksMax) by one block.
+// In-place exclusive scan of a short array by one block (four items per thread and sweep).
 __global__ void __launch_bounds__(1024) rs_scan_kernel(uint32_t *a, int n) {
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t carry_s;
   if (threadIdx.x == 0) carry_s = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  for (int base = 0; base < n; base += 1024) {
-    int i = base + threadIdx.x;
-    uint32_t v = i < n ? a[i] : 0u;
-    uint32_t inc = v;
+  for (int base = 0; base < n; base += 4096) {
+    int i = base + threadIdx.x * 4;
+    uint32_t v[4], sum = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[j] = i + j < n ? a[i + j] : 0u;
+      sum += v[j];
+    }
+    uint32_t inc = sum;
     for (int o = 1; o < 32; o <<= 1) {
       uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
       if (lane >= o) inc += u;
@@ -67,106 +77,212 @@ __global__ void __launch_bounds__(1024) rs_scan_kernel(uint32_t *a, int n) {
       warp_tot[lane] = ti - t;  // exclusive prefix of the warp totals
     }
     __syncthreads();
-    uint32_t carry = carry_s;
-    uint32_t excl = carry + warp_tot[w] + inc - v;
-    if (i < n) a[i] = excl;
+    uint32_t run = carry_s + warp_tot[w] + inc - sum;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (i + j < n) a[i + j] = run;
+      run += v[j];
+    }
     __syncthreads();
-    if (threadIdx.x == 1023) carry_s = excl + v;
+    if (threadIdx.x == 1023) carry_s = run;
     __syncthreads();
   }
 }
 
-__global__ void __launch_bounds__(RS_THREADS)
-rs_scatter_kernel(const uint32_t *__restrict__ kin, const uint32_t *__restrict__ vin,
-                  uint32_t *__restrict__ kout, uint32_t *__restrict__ vout, int64_t n,
-                  int64_t per_block, int shift, uint32_t mask, const uint32_t *__restrict__ offs,
-                  int nb) {
-  __shared__ uint32_t wc[RS_WARPS][RS_RADIX];
-  __shared__ uint32_t off[RS_RADIX];
+// One key stream and NP payload streams of a sort pass.  pin[q] == nullptr: payload q is the
+// position of the item in the input (a sort that starts from the identity permutation).
+template <int NP>
+struct SortIO {
+  const uint32_t *kin;
+  uint32_t *kout;
+  const uint32_t *pin[NP];
+  uint32_t *pout[NP];
+};
+
+constexpr size_t rs_scatter_smem(int np) {
+  return sizeof(uint32_t) * ((size_t)RS_WARPS * RS_RADIX + 2 * RS_RADIX + 32 + (size_t)(1 + np) * RS_TILE);
+}
+
+// Stable scatter of one pass.  Each block owns a contiguous range of the input and walks it in
+// tiles.  Within a tile every item gets its rank among the tile's items of the same digit in
+// input order (warp match + per-warp digit counters + a scan over the warps); the tile is
+// then put in digit order in shared memory, so that the copy to global memory writes each
+// digit's items to consecutive addresses from consecutive threads.
+template <int NP>
+__global__ void __launch_bounds__(RS_THREADS, 2)
+rs_scatter_kernel(SortIO<NP> io, int64_t n, int64_t per_block, int shift, uint32_t mask,
+                  const uint32_t *__restrict__ offs, int nb) {
+  extern __shared__ uint32_t rs_sm[];
+  uint32_t(*wc)[RS_RADIX] = reinterpret_cast<uint32_t(*)[RS_RADIX]>(rs_sm);
+  uint32_t *lstart = rs_sm + RS_WARPS * RS_RADIX;  // first staged slot of each digit
+  uint32_t *gadj = lstart + RS_RADIX;              // global position of a staged slot = gadj[digit] + slot
+  uint32_t *wtot = gadj + RS_RADIX;
+  uint32_t *skey = wtot + 32;
+  uint32_t *sval = skey + RS_TILE;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const uint32_t lt = (1u << lane) - 1u;
-  for (int d = threadIdx.x; d < RS_RADIX; d += RS_THREADS) off[d] = offs[(size_t)d * nb + blockIdx.x];
+  // thread d keeps the running global offset of digit d for this block
+  uint32_t run_off = (uint32_t)threadIdx.x <= mask ? offs[(size_t)threadIdx.x * nb + blockIdx.x] : 0u;
   int64_t lo = (int64_t)blockIdx.x * per_block;
   int64_t hi = lo + per_block < n ? lo + per_block : n;
+  // The keys of the next tile are fetched while this tile is ranked and written, and the
+  // payload words of this tile while it is ranked, so that no load is waited for in place.
+  uint32_t nkey[RS_ITEMS];
+#pragma unroll
+  for (int it = 0; it < RS_ITEMS; ++it) {
+    int64_t p = lo + (int64_t)w * 32 * RS_ITEMS + it * 32 + lane;
+    nkey[it] = p < hi ? io.kin[p] : 0u;
+  }
   for (int64_t tile = lo; tile < hi; tile += RS_TILE) {
     for (int d = lane; d < RS_RADIX; d += 32) wc[w][d] = 0;
-    __syncthreads();  // also orders the initial off[] load and the previous tile's reads
-    uint32_t key[RS_ITEMS], val[RS_ITEMS], rank[RS_ITEMS], dig[RS_ITEMS];
+    __syncwarp();
+    uint32_t key[RS_ITEMS], rank[RS_ITEMS], pay[NP][RS_ITEMS];
     const int64_t wbase = tile + (int64_t)w * 32 * RS_ITEMS;
 #pragma unroll
     for (int it = 0; it < RS_ITEMS; ++it) {
-      int64_t p = wbase + it * 32 + lane;
-      bool ok = p < hi;
-      key[it] = ok ? kin[p] : 0u;
-      val[it] = ok ? (vin ? vin[p] : (uint32_t)p) : 0u;
-      dig[it] = ok ? ((key[it] >> shift) & mask) : 0xffffffffu;
+      key[it] = nkey[it];
+      int64_t p = wbase + RS_TILE + it * 32 + lane;
+      nkey[it] = p < hi ? io.kin[p] : 0u;
+    }
+#pragma unroll
+    for (int q = 0; q < NP; ++q) {
+#pragma unroll
+      for (int it = 0; it < RS_ITEMS; ++it) {
+        int64_t p = wbase + it * 32 + lane;
+        pay[q][it] = (p < hi && io.pin[q]) ? io.pin[q][p] : (uint32_t)p;
+      }
     }
 #pragma unroll
     for (int it = 0; it < RS_ITEMS; ++it) {
-      uint32_t peers = __match_any_sync(0xffffffffu, dig[it]);
+      const bool ok = wbase + it * 32 + lane < hi;
+      const uint32_t dig = ok ? ((key[it] >> shift) & mask) : 0xffffffffu;
+      uint32_t peers = __match_any_sync(0xffffffffu, dig);
       int leader = __ffs(peers) - 1;
       uint32_t base = 0;
-      if (lane == leader && dig[it] != 0xffffffffu) {
-        base = wc[w][dig[it]];
-        wc[w][dig[it]] = base + __popc(peers);
+      if (lane == leader && ok) {
+        base = wc[w][dig];
+        wc[w][dig] = base + __popc(peers);
       }
       base = __shfl_sync(0xffffffffu, base, leader);
       rank[it] = base + __popc(peers & lt);
       __syncwarp();
     }
     __syncthreads();
-    {  // thread d: exclusive scan of digit d over the warps, shifted by the running offset
-      int d = threadIdx.x;
-      uint32_t run = off[d];
+    // thread d < RS_RADIX: scan digit d over the warps, then the digit totals over d
+    uint32_t tot = 0, inc = 0;
+    if (threadIdx.x < RS_RADIX) {
+      const int d = threadIdx.x;
 #pragma unroll
       for (int ww = 0; ww < RS_WARPS; ++ww) {
         uint32_t c = wc[ww][d];
-        wc[ww][d] = run;
-        run += c;
+        wc[ww][d] = tot;
+        tot += c;
       }
-      off[d] = run;
+      inc = tot;
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += u;
+      }
+      if (lane == 31) wtot[w] = inc;
+    }
+    __syncthreads();
+    if (threadIdx.x < RS_RADIX) {
+      uint32_t pre = 0;
+      for (int ww = 0; ww < w; ++ww) pre += wtot[ww];
+      const uint32_t ls = pre + inc - tot;
+      lstart[threadIdx.x] = ls;
+      gadj[threadIdx.x] = run_off - ls;
+      run_off += tot;
     }
     __syncthreads();
 #pragma unroll
     for (int it = 0; it < RS_ITEMS; ++it) {
-      if (dig[it] != 0xffffffffu) {
-        uint32_t pos = wc[w][dig[it]] + rank[it];
-        kout[pos] = key[it];
-        vout[pos] = val[it];
+      const int64_t p = wbase + it * 32 + lane;
+      if (p < hi) {
+        const uint32_t dig = (key[it] >> shift) & mask;
+        const uint32_t slot = lstart[dig] + wc[w][dig] + rank[it];
+        skey[slot] = key[it];
+#pragma unroll
+        for (int q = 0; q < NP; ++q) sval[q * RS_TILE + slot] = pay[q][it];
       }
+    }
+    __syncthreads();
+    const int cnt = (int)(hi - tile < RS_TILE ? hi - tile : RS_TILE);
+#pragma unroll 4
+    for (int i = threadIdx.x; i < cnt; i += RS_THREADS) {
+      const uint32_t k = skey[i];
+      const uint32_t g = gadj[(k >> shift) & mask] + (uint32_t)i;
+      io.kout[g] = k;
+#pragma unroll
+      for (int q = 0; q < NP; ++q) io.pout[q][g] = sval[q * RS_TILE + i];
     }
     __syncthreads();
   }
 }
 
-// Stable sort of n pairs on key bits [0, nbits).  Reads (kin, vin) (vin == nullptr: the
-// payload is the position), ping-pongs between (kA, vA) and (kB, vB); *kres / *vres point at
-// the buffers holding the result.
-cudaError_t radix_sort_pairs(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits,
-                             LayoutScratch &s, cudaStream_t st, uint32_t **kres, uint32_t **vres) {
+// The two buffer sets a sort ping-pongs between.
+struct SortSet {
+  uint32_t *k;
+  uint32_t *p[RS_MAXP];
+};
+inline SortSet set_a(const LayoutScratch &s) { return SortSet{s.kA, {s.vA, s.wA, s.xA}}; }
+inline SortSet set_b(const LayoutScratch &s) { return SortSet{s.kB, {s.vB, s.wB, s.xB}}; }
+inline bool in_set(const SortSet &x, const void *ptr) {
+  if (!ptr) return false;
+  if (ptr == x.k) return true;
+  for (int q = 0; q < RS_MAXP; ++q)
+    if (ptr == x.p[q]) return true;
+  return false;
+}
+
+// Stable sort of n items (key + NP payload words) on key bits [0, nbits).  The passes
+// ping-pong between the two buffer sets of the scratch, starting with the set that holds none
+// of the inputs; where kfin / pfin[q] is not null the last pass writes that stream there
+// instead (it must not alias an input of that pass).  *kres / pres[q] receive the location of
+// each result stream.
+template <int NP>
+cudaError_t radix_sort_multi(const uint32_t *kin, const uint32_t *const *pin, int64_t n, int nbits,
+                             LayoutScratch &s, cudaStream_t st, uint32_t *kfin, uint32_t *const *pfin,
+                             uint32_t **kres, uint32_t **pres) {
+  static_assert(NP >= 1 && NP <= RS_MAXP, "payload count");
   int npass = (nbits + 7) / 8;
   if (npass < 1) npass = 1;
   int64_t tiles = (n + RS_TILE - 1) / RS_TILE;
   int nb = (int)(tiles < kSortBlocksMax ? tiles : kSortBlocksMax);
   if (nb < 1) nb = 1;
   int64_t per_block = ((tiles + nb - 1) / nb) * RS_TILE;
-  const uint32_t *ck = kin, *cv = vin;
-  uint32_t *ok = s.kA, *ov = s.vA;
+  const SortSet A = set_a(s), B = set_b(s);
+  bool inA = in_set(A, kin), inB = in_set(B, kin);
+  for (int q = 0; q < NP; ++q) {
+    inA = inA || in_set(A, pin[q]);
+    inB = inB || in_set(B, pin[q]);
+  }
+  if (inA && inB) return cudaErrorInvalidValue;
+  CK(cudaFuncSetAttribute(rs_scatter_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                          (int)rs_scatter_smem(NP)));
+  SortSet out = inA ? B : A, other = inA ? A : B;
+  SortIO<NP> io;
+  io.kin = kin;
+  for (int q = 0; q < NP; ++q) io.pin[q] = pin[q];
   int shift = 0;
   for (int p = 0; p < npass; ++p) {
     int bits = (nbits - shift + (npass - p) - 1) / (npass - p);  // spread the bits evenly
     if (bits < 1) bits = 1;
     uint32_t mask = (1u << bits) - 1u;
-    rs_hist_kernel<<<nb, RS_THREADS, 0, st>>>(ck, n, per_block, shift, mask, s.hist, nb);
-    rs_scan_kernel<<<1, 1024, 0, st>>>(s.hist, RS_RADIX * nb);
-    rs_scatter_kernel<<<nb, RS_THREADS, 0, st>>>(ck, cv, ok, ov, n, per_block, shift, mask, s.hist, nb);
+    const bool last = p == npass - 1;
+    io.kout = (last && kfin) ? kfin : out.k;
+    for (int q = 0; q < NP; ++q) io.pout[q] = (last && pfin && pfin[q]) ? pfin[q] : out.p[q];
+    rs_hist_kernel<<<nb, RS_HIST_THREADS, 0, st>>>(io.kin, n, per_block, shift, mask, s.hist, nb);
+    rs_scan_kernel<<<1, 1024, 0, st>>>(s.hist, (int)(mask + 1) * nb);
+    rs_scatter_kernel<NP><<<nb, RS_THREADS, rs_scatter_smem(NP), st>>>(io, n, per_block, shift, mask, s.hist, nb);
     CK(cudaGetLastError());
-    ck = ok; cv = ov;
-    if (ok == s.kA) { ok = s.kB; ov = s.vB; } else { ok = s.kA; ov = s.vA; }
+    io.kin = io.kout;
+    for (int q = 0; q < NP; ++q) io.pin[q] = io.pout[q];
+    SortSet tmp = out; out = other; other = tmp;
     shift += bits;
   }
-  *kres = const_cast<uint32_t *>(ck);
-  *vres = const_cast<uint32_t *>(cv);
+  *kres = const_cast<uint32_t *>(io.kin);
+  for (int q = 0; q < NP; ++q) pres[q] = const_cast<uint32_t *>(io.pin[q]);
   return cudaSuccess;
 }
 
@@ -218,7 +334,7 @@ cudaError_t exclusive_scan_u32(const uint32_t *in, uint32_t *out, int64_t n, Lay
   return cudaGetLastError();
 }
 
-// ---- checks, gathers, pointer arrays ------------------------------------------------------------
+// ---- checks, copies, pointer arrays ------------------------------------------------------------
 __global__ void check_coo_kernel(const int32_t *__restrict__ rows, const int32_t *__restrict__ cols,
                                  int64_t nnz, int32_t m, int32_t n, int32_t *flags) {
   int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -244,14 +360,6 @@ __global__ void check_dup_kernel(const uint32_t *__restrict__ rowkey, const int3
   for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x + 1; p < nnz; p += stride)
     if (rowkey[p] == rowkey[p - 1] && col_idx[p] == col_idx[p - 1]) dup = true;
   if (dup) flags[FLAG_DUP] = 1;
-}
-
-template <typename TI, typename TO>
-__global__ void gather_kernel(const TI *__restrict__ src, const uint32_t *__restrict__ pos, TO *__restrict__ dst,
-                              int64_t n) {
-  int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += stride)
-    dst[p] = (TO)src[pos[p]];
 }
 
 template <typename TI, typename TO>
@@ -341,30 +449,25 @@ cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t 
   if (h_flags[FLAG_UNSORTED] && (t->cfg.flags & TSID_INPUT_ROW_SORTED)) return cudaSuccess;
 
   const int g = grid_for(nnz, 256);
-  uint32_t *rowkey = reinterpret_cast<uint32_t *>(t->val_csc);  // parked here until val_csc is written
+  const uint32_t *rowkey = reinterpret_cast<const uint32_t *>(d_rows);  // row of each entry in CSR order
   if (nnz > 0) {
     if (!h_flags[FLAG_UNSORTED]) {
       // already in (row, col) order: CSR is the input
       copy_kernel<int32_t, int32_t><<<g, 256, 0, st>>>(d_cols, t->col_idx, nnz);
       copy_kernel<float, float><<<g, 256, 0, st>>>(d_vals, t->val_csr, nnz);
-      copy_kernel<int32_t, uint32_t><<<g, 256, 0, st>>>(d_rows, rowkey, nnz);
     } else {
       h_flags[FLAG_DUP] = 0;  // the adjacent-pair test of check_coo only holds for sorted input
       CK(cudaMemsetAsync(t->flags + FLAG_DUP, 0, sizeof(int32_t), st));
-      uint32_t *k1, *v1, *k2, *v2;
-      // stable by column, then stable by row  =>  (row, col, input position) order
-      CK(radix_sort_pairs(reinterpret_cast<const uint32_t *>(d_cols), nullptr, nnz, bits_for(n - 1), s, st, &k1, &v1));
-      // keys for the second sort: row of each entry in the current order
-      // (the sort first writes to (kA, vA), so its input must sit in the B buffers; the sorted
-      // column keys in k1 are no longer needed)
-      (void)k1;
-      uint32_t *gk = s.kB;
-      gather_kernel<int32_t, uint32_t><<<g, 256, 0, st>>>(d_rows, v1, gk, nnz);
-      if (v1 == s.vA) { copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(v1, s.vB, nnz); v1 = s.vB; }
-      CK(radix_sort_pairs(gk, v1, nnz, bits_for(m - 1), s, st, &k2, &v2));
-      gather_kernel<int32_t, int32_t><<<g, 256, 0, st>>>(d_cols, v2, t->col_idx, nnz);
-      gather_kernel<float, float><<<g, 256, 0, st>>>(d_vals, v2, t->val_csr, nnz);
-      copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(k2, rowkey, nnz);
+      // stable by column, then stable by row  =>  (row, col, input position) order; the other
+      // index and the value travel with the key, so nothing is gathered afterwards
+      uint32_t *k1, *p1[2], *k2, *p2[2];
+      const uint32_t *in1[2] = {reinterpret_cast<const uint32_t *>(d_rows), reinterpret_cast<const uint32_t *>(d_vals)};
+      CK(radix_sort_multi<2>(reinterpret_cast<const uint32_t *>(d_cols), in1, nnz, bits_for(n - 1), s, st, nullptr,
+                             nullptr, &k1, p1));
+      const uint32_t *in2[2] = {k1, p1[1]};
+      uint32_t *fin2[2] = {reinterpret_cast<uint32_t *>(t->col_idx), reinterpret_cast<uint32_t *>(t->val_csr)};
+      CK(radix_sort_multi<2>(p1[0], in2, nnz, bits_for(m - 1), s, st, nullptr, fin2, &k2, p2));
+      rowkey = k2;
       if (t->cfg.flags & TSID_VALIDATE) check_dup_kernel<<<g, 256, 0, st>>>(rowkey, t->col_idx, nnz, t->flags);
     }
     CK(cudaGetLastError());
@@ -372,14 +475,14 @@ cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t 
   ptr_from_sorted_kernel<<<grid_for(nnz + 1, 256), 256, 0, st>>>(rowkey, nnz, m, t->row_ptr);
   CK(cudaGetLastError());
 
-  // CSC: stable sort of the CSR positions by column
+  // CSC: stable sort of the CSR entries by column, carrying (CSR position, row, value)
   if (nnz > 0) {
-    uint32_t *k3, *v3;
-    CK(radix_sort_pairs(reinterpret_cast<const uint32_t *>(t->col_idx), nullptr, nnz, bits_for(n - 1), s, st, &k3, &v3));
-    copy_kernel<uint32_t, uint32_t><<<g, 256, 0, st>>>(v3, t->perm, nnz);
+    uint32_t *k3, *p3[3];
+    const uint32_t *in3[3] = {nullptr, rowkey, reinterpret_cast<const uint32_t *>(t->val_csr)};
+    uint32_t *fin3[3] = {t->perm, reinterpret_cast<uint32_t *>(t->row_idx), reinterpret_cast<uint32_t *>(t->val_csc)};
+    CK(radix_sort_multi<3>(reinterpret_cast<const uint32_t *>(t->col_idx), in3, nnz, bits_for(n - 1), s, st, nullptr,
+                           fin3, &k3, p3));
     ptr_from_sorted_kernel<<<grid_for(nnz + 1, 256), 256, 0, st>>>(k3, nnz, n, t->col_ptr);
-    gather_kernel<uint32_t, int32_t><<<g, 256, 0, st>>>(rowkey, t->perm, t->row_idx, nnz);
-    gather_kernel<float, float><<<g, 256, 0, st>>>(t->val_csr, t->perm, t->val_csc, nnz);  // overwrites rowkey
     CK(cudaGetLastError());
   } else {
     ptr_from_sorted_kernel<<<1, 256, 0, st>>>(nullptr, 0, n, t->col_ptr);
@@ -421,7 +524,8 @@ cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutSc
 // The sort and the scan, for the other translation units (template sampling).
 cudaError_t sort_pairs_u32(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits, LayoutScratch &s,
                            cudaStream_t st, uint32_t **kres, uint32_t **vres) {
-  return radix_sort_pairs(kin, vin, n, nbits, s, st, kres, vres);
+  const uint32_t *pin[1] = {vin};
+  return radix_sort_multi<1>(kin, pin, n, nbits, s, st, nullptr, nullptr, kres, vres);
 }
 cudaError_t scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch &s, cudaStream_t st) {
   return exclusive_scan_u32(in, out, n, s, st);

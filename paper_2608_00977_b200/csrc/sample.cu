@@ -103,6 +103,7 @@ SampleCarve carve(void *base, int32_t n, int64_t nnz) {
   c.dflags = cv.take<int32_t>(FLAG_COUNT);
   c.ls.kA = cv.take<uint32_t>(nn); c.ls.kB = cv.take<uint32_t>(nn);
   c.ls.vA = cv.take<uint32_t>(nn); c.ls.vB = cv.take<uint32_t>(nn);
+  c.ls.wA = c.ls.wB = c.ls.xA = c.ls.xB = nullptr;
   c.ls.hist = cv.take<uint32_t>(256 * (size_t)kSortBlocksMax);
   c.ls.scanA = c.ls.scanB = c.ls.scanC = nullptr;
   c.ls.blocksums = cv.take<uint32_t>(kScanBlocksMax);

@@ -102,19 +102,20 @@ struct Carver {
 
 // Transient buffers of the layout pass (also carved from the workspace).
 struct LayoutScratch {
-  uint32_t *kA, *kB, *vA, *vB;  // [nnz] each
+  uint32_t *kA, *kB, *vA, *vB;  // [nnz] each: key and first payload of the two sort buffer sets
+  uint32_t *wA, *wB, *xA, *xB;  // [nnz] each or null: second and third payload (layout pass only)
   uint32_t *hist;               // [256 * kSortBlocks]
   uint32_t *scanA, *scanB, *scanC;  // [max(m,n)+1] each
   uint32_t *blocksums;          // [kScanBlocksMax]
 };
-constexpr int kSortBlocksMax = 2048;
+constexpr int kSortBlocksMax = 148 * 6;
 constexpr int kScanBlocksMax = 1 << 20;
 
 cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols,
                          const float *d_vals, LayoutScratch &s, int32_t h_flags[FLAG_COUNT]);
 cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutScratch &s);
 // stable LSD radix sort of (key, payload) pairs on key bits [0, nbits) (vin == nullptr: payload = position);
-// ping-pongs between (s.kA, s.vA) and (s.kB, s.vB), the input must not live in kA / vA
+// ping-pongs between (s.kA, s.vA) and (s.kB, s.vB), first writing the pair that holds no input
 cudaError_t sort_pairs_u32(const uint32_t *kin, const uint32_t *vin, int64_t n, int nbits, LayoutScratch &s,
                            cudaStream_t st, uint32_t **kres, uint32_t **vres);
 // out[0..n) = exclusive scan of in[0..n), out[n] = total; in[n] must be 0; in may alias out
