@@ -397,7 +397,7 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step) {
   if (!t) return TSID_ERR_INVALID_ARG;
   if (h_path) *h_path = t->path;
-  if (h_launches_per_step) *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? 4 : sparse_launches_per_step(t);
+  if (h_launches_per_step) *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? dense_launches_per_step(t) : sparse_launches_per_step(t);
   return TSID_OK;
 }
 

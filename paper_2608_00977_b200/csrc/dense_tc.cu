@@ -3,21 +3,25 @@
 // is only a mask).  For templates dense enough that this really is a dense contraction:
 //
 //   pass A (CTA per block of 128 rows i, loop over blocks of 128 columns j):
-//       S = P_blk Q_blk^T            tcgen05.mma, bf16 operands from shared memory (TMA), fp32 in TMEM
+//       S = P_blk Q_blk^T            tcgen05.mma, A = the CTA's own factor block held in TMEM for the whole
+//                                    kernel, B = the Q tile in shared memory (TMA), fp32 accumulator in TMEM
 //       E = M .* (R - S)             epilogue warps: S from TMEM, the R tile (fp16, NaN = unobserved) from
-//                                    shared memory (TMA); E goes back to TMEM as packed bf16
+//                                    shared memory (TMA); E goes back to TMEM as packed bf16, in place
 //       G_P_blk += E Q_blk           tcgen05.mma with A = E read from TMEM, accumulating in TMEM over the
 //                                    whole j loop
 //   pass B: the same kernel on (Q, P, R^T) gives G_Q.
 //
 // S is computed in both passes (four GEMMs instead of three) so that each gradient block has one
-// owner CTA and a fixed summation order: no atomics, no partial buffers.  A 128x128x16 MMA with both
-// operands in shared memory reads 128 B per clock, the whole shared-memory bandwidth of an SM; keeping
-// E in TMEM removes its round trip through shared memory and halves what the second MMA reads there.
-// The Y tile (128 rows j x K columns, 128-byte-swizzled as TMA writes it) serves both products: K-major
-// as B of the first (contraction over the factor index) and MN-major as B of the second (contraction
-// over j), so no transposed copy of the factors exists.  Every mbarrier wait is bounded by a cycle budget; on
-// expiry the CTA raises FLAG_TIMEOUT, stops issuing, and still frees its TMEM before it returns.
+// owner and a fixed summation order: no atomics.  Both products take their A operand from TMEM: a
+// 128 x 128 x 16 MMA whose A comes from shared memory was measured at ~129 clocks on this part against
+// ~73 with A in TMEM (64 is the tensor pipe's own time), so the owner block is copied to TMEM once
+// and E never leaves it.  The Y tile (128 rows j x K columns, 128-byte-swizzled as TMA writes it)
+// serves both products: K-major as B of the first (contraction over the factor index) and MN-major as
+// B of the second (contraction over j), so no transposed copy of the factors exists.  When there are
+// fewer row blocks than SMs the column range is split over several CTAs per row block; each writes its
+// own partial gradient block and a small kernel adds them in a fixed order.  Every mbarrier wait is
+// bounded by a cycle budget; on expiry the CTA raises FLAG_TIMEOUT, stops issuing, and still frees its
+// TMEM before it returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -29,6 +33,7 @@ namespace tsid {
 
 struct DenseState {
   __half *R = nullptr, *RT = nullptr;              // [m*n], [n*m]; NaN = not observed
+  float *gpart = nullptr;                          // [(MAX_SPLIT - 1) * max(m, n) * k] partial gradient blocks
   CUtensorMap tmP, tmQ, tmR, tmRT;
 };
 
@@ -40,8 +45,8 @@ namespace {
     if (e_ != cudaSuccess) return e_; \
   } while (0)
 
-constexpr int BLK = 128;                 // tile edge (rows of X per CTA, rows of Y per iteration)
-constexpr int NSTAGE = 3;                // stages of the Y and R tiles
+constexpr int BLK = 128;                 // tile edge (rows of one X half, rows of Y per iteration)
+constexpr int MAX_SPLIT = 4;             // CTAs sharing one row block (each takes a range of column blocks)
 constexpr long long WAIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz: bound of every wait
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -82,15 +87,6 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]   (A: lane = row, 32-bit column = two consecutive bf16 along K)
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
@@ -156,36 +152,43 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n) {
 
 template <int K>
 struct Smem {
+  static constexpr int NSY = 3;                   // stages of the Y tile ring
+  static constexpr int NSR = 4;                   // stages of the R tile ring
   static constexpr int XB = BLK * 128;            // one 64-column block of a 128-row tile: 16 KB
-  static constexpr int X_BYTES = (K / 64) * XB;   // X block (128 x K bf16)
   static constexpr int Y_BYTES = (K / 64) * XB;   // Y block (128 x K bf16)
   static constexpr int R_BYTES = 2 * XB;          // R tile (128 x 128 fp16)
-  static constexpr int STAGE_BYTES = Y_BYTES + R_BYTES;
-  static constexpr int OFF_X = 0;
-  static constexpr int OFF_Y = OFF_X + X_BYTES;
-  static constexpr int OFF_R = OFF_Y + NSTAGE * Y_BYTES;
-  static constexpr int OFF_BAR = OFF_R + NSTAGE * R_BYTES;
+  static constexpr int OFF_Y = 0;
+  static constexpr int OFF_R = OFF_Y + NSY * Y_BYTES;
+  static constexpr int OFF_BAR = OFF_R + NSR * R_BYTES;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // barriers + slack for 1024-byte alignment
+  // barrier indices
+  static constexpr int B_XFULL = 0, B_YFULL = 1, B_YEMPTY = B_YFULL + NSY, B_RFULL = B_YEMPTY + NSY,
+                       B_REMPTY = B_RFULL + NSR, B_SFULL = B_REMPTY + NSR, B_EFULL = B_SFULL + 2,
+                       B_GFULL = B_EFULL + 2, B_COUNT = B_GFULL + 1;
+  static_assert(B_COUNT * 8 <= 192, "barriers overlap the TMEM address slot");
+  static_assert(TOTAL <= 232448, "shared memory of one CTA");
 };
 
-enum { B_XFULL = 0, B_QFULL = 1, B_QEMPTY = 1 + NSTAGE, B_SFULL = 1 + 2 * NSTAGE, B_SEMPTY = B_SFULL + 2, B_EFULL = B_SFULL + 4,
-       B_EEMPTY = B_SFULL + 6, B_GFULL = B_SFULL + 8, B_COUNT = B_SFULL + 9 };
-static_assert(B_COUNT * 8 <= 192, "barriers overlap the TMEM address slot");
-
-// TMEM columns (512 allocated): S tiles 0..127 and 128..255 (fp32), G block 256..383 (fp32, K used),
-// E tiles 384..447 and 448..511 (packed bf16: 64 columns hold 128 values per row).
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_G = 256, TM_E0 = 384, TM_E1 = 448;
+// TMEM columns (512 allocated): the CTA's X block as packed bf16 at 0 (K / 2 columns used), S tiles at
+// 64 and 192 (fp32; the epilogue overwrites the first 32 columns of each 64-column half with the packed
+// bf16 E values of that half), G block at 320 (fp32, K columns used).
+constexpr uint32_t TM_X = 0, TM_S0 = 64, TM_S1 = 192, TM_G = 320;
 
 // One pass: G_X[rows_x x K] = (M .* (R - X Y^T)) Y, R given as fp16 [rows_x][rows_y] with NaN = unobserved.
+// CTA (ib, sp) owns rows [128 ib, 128 ib + 128) of X and the column blocks [NJ sp / nsplit,
+// NJ (sp + 1) / nsplit) of Y; split 0 writes to G, split sp > 0 to its partial buffer.  Work item w is
+// the w-th column block of the CTA; it uses S buffer and epilogue team w & 1, so the TMEM round trips of
+// one item overlap with the tensor work of the next.
 // Warps: 0 = TMA producer, 1 = MMA issuer (one thread), 2..17 = two epilogue teams of eight warps (two
-// warps per TMEM lane quarter; a thread owns one row of the tile and half of its columns).  Team 0 takes
-// the even column blocks (S0 / E0 / stage 0), team 1 the odd ones, so that the TMEM round trips of one
-// tile overlap with the arithmetic of the next.
+// warps per TMEM lane quarter; a thread owns one row of the tile and half of its columns).
+// TMEM reuse needs no barrier of its own: the MMAs of one CTA execute in issue order, and the first
+// product of item w + 2 is issued after the second product of item w, which is the last reader of that
+// S / E buffer.
 template <int K>
 __global__ void __launch_bounds__(576, 1)
-dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-                  const __grid_constant__ CUtensorMap tmR, int rows_y,
-                  float *__restrict__ G, int32_t *__restrict__ flags) {
+dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ CUtensorMap tmY,
+                  const __grid_constant__ CUtensorMap tmR, int rows_x, int rows_y, int nsplit,
+                  float *__restrict__ G, float *__restrict__ Gpart, int32_t *__restrict__ flags) {
   using L = Smem<K>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;   // tiles need 1024-byte alignment
@@ -195,15 +198,19 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ib = blockIdx.x;
+  const int ib = blockIdx.x / nsplit, sp = blockIdx.x % nsplit;
+  const int row0 = ib * BLK;
   const int NJ = rows_y / BLK;
+  const int jb0 = (int)((long long)NJ * sp / nsplit), jb1 = (int)((long long)NJ * (sp + 1) / nsplit);
+  const int NW = jb1 - jb0;                // work items of this CTA
+  float *Gout = sp == 0 ? G : Gpart + (size_t)(sp - 1) * rows_x * K;
 
   if (threadIdx.x == 0) {
-    mbar_init(bar(B_XFULL), 1);
-    for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(B_QFULL + s), 1); mbar_init(bar(B_QEMPTY + s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_SFULL + b), 1); mbar_init(bar(B_SEMPTY + b), 8); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_EFULL + b), 8); mbar_init(bar(B_EEMPTY + b), 1); }
-    mbar_init(bar(B_GFULL), 1);
+    mbar_init(bar(L::B_XFULL), 8);
+    for (int s = 0; s < L::NSY; ++s) { mbar_init(bar(L::B_YFULL + s), 1); mbar_init(bar(L::B_YEMPTY + s), 1); }
+    for (int s = 0; s < L::NSR; ++s) { mbar_init(bar(L::B_RFULL + s), 1); mbar_init(bar(L::B_REMPTY + s), 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar(L::B_SFULL + b), 1); mbar_init(bar(L::B_EFULL + b), 8); }
+    mbar_init(bar(L::B_GFULL), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -214,25 +221,26 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const uint32_t tmX = tmem + TM_X;
   const uint32_t tmS[2] = {tmem + TM_S0, tmem + TM_S1};
-  const uint32_t tmE[2] = {tmem + TM_E0, tmem + TM_E1};
   const uint32_t tmG = tmem + TM_G;
   bool ok = true;
 
   if (warp == 0) {
     // ---- TMA producer ---------------------------------------------------------------------------
     if (lane == 0) {
-      mbar_expect_tx(bar(B_XFULL), L::X_BYTES);
-      for (int h = 0; h < K / 64; ++h) tma_load_2d(sm0 + L::OFF_X + h * L::XB, &tmX, bar(B_XFULL), h * 64, ib * BLK);
-      for (int jb = 0; jb < NJ && ok; ++jb) {
-        const int st = jb % NSTAGE;
-        if (jb >= NSTAGE) ok = mbar_wait(bar(B_QEMPTY + st), ((jb / NSTAGE) - 1) & 1);
+      for (int w = 0; w < NW && ok; ++w) {
+        const int jb = jb0 + w, ys = w % L::NSY, rs = w % L::NSR;
+        if (w >= L::NSY) ok = mbar_wait(bar(L::B_YEMPTY + ys), ((w / L::NSY) - 1) & 1);
         if (!ok) break;
-        mbar_expect_tx(bar(B_QFULL + st), L::STAGE_BYTES);
-        for (int h = 0; h < K / 64; ++h)
-          tma_load_2d(sm0 + L::OFF_Y + st * L::Y_BYTES + h * L::XB, &tmY, bar(B_QFULL + st), h * 64, jb * BLK);
-        for (int h = 0; h < 2; ++h)
-          tma_load_2d(sm0 + L::OFF_R + st * L::R_BYTES + h * L::XB, &tmR, bar(B_QFULL + st), jb * BLK + h * 64, ib * BLK);
+        mbar_expect_tx(bar(L::B_YFULL + ys), L::Y_BYTES);
+        for (int c = 0; c < K / 64; ++c)
+          tma_load_2d(sm0 + L::OFF_Y + ys * L::Y_BYTES + c * L::XB, &tmY, bar(L::B_YFULL + ys), c * 64, jb * BLK);
+        if (w >= L::NSR) ok = mbar_wait(bar(L::B_REMPTY + rs), ((w / L::NSR) - 1) & 1);
+        if (!ok) break;
+        mbar_expect_tx(bar(L::B_RFULL + rs), L::R_BYTES);
+        for (int c = 0; c < 2; ++c)
+          tma_load_2d(sm0 + L::OFF_R + rs * L::R_BYTES + c * L::XB, &tmR, bar(L::B_RFULL + rs), jb * BLK + c * 64, row0);
       }
     }
     __syncwarp();
@@ -240,38 +248,36 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     // ---- MMA issuer -----------------------------------------------------------------------------
     if (lane == 0) {
       constexpr uint32_t ID1 = idesc_bf16(BLK), ID2 = idesc_bf16(K) | (1u << 16);   // second product: B is MN-major
-      auto mma1 = [&](int jb) -> bool {
-        const int st = jb % NSTAGE, b = jb & 1;
-        if (!mbar_wait(bar(B_QFULL + st), (jb / NSTAGE) & 1)) return false;
-        if (jb >= 2 && !mbar_wait(bar(B_SEMPTY + b), ((jb >> 1) - 1) & 1)) return false;
+      auto mma1 = [&](int w) -> bool {
+        const int ys = w % L::NSY, b = w & 1;
+        if (!mbar_wait(bar(L::B_YFULL + ys), (w / L::NSY) & 1)) return false;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < K / 16; ++ks) {
+        for (int ks = 0; ks < K / 16; ++ks) {   // A: 16 factor columns = 8 TMEM columns of the X block
           const uint32_t off = (ks / 4) * L::XB + (ks % 4) * 32;
-          tc_mma_ss(tmS[b], smem_desc(sm0 + L::OFF_X + off), smem_desc(sm0 + L::OFF_Y + st * L::Y_BYTES + off), ID1,
-                    ks > 0);
+          tc_mma_ts(tmS[b], tmX + ks * 8, smem_desc(sm0 + L::OFF_Y + ys * L::Y_BYTES + off), ID1, ks > 0);
         }
-        tc_commit(bar(B_SFULL + b));
+        tc_commit(bar(L::B_SFULL + b));
         return true;
       };
-      ok = mbar_wait(bar(B_XFULL), 0);
-      if (ok) ok = mma1(0);
-      for (int jb = 0; jb < NJ && ok; ++jb) {
-        const int st = jb % NSTAGE, b = jb & 1;
-        if (jb + 1 < NJ) ok = mma1(jb + 1);
-        if (ok) ok = mbar_wait(bar(B_EFULL + b), (jb >> 1) & 1);
+      ok = mbar_wait(bar(L::B_XFULL), 0);
+      if (ok && NW > 0) ok = mma1(0);
+      for (int w = 0; w < NW && ok; ++w) {
+        const int ys = w % L::NSY, b = w & 1;
+        if (w + 1 < NW) ok = mma1(w + 1);
+        if (ok) ok = mbar_wait(bar(L::B_EFULL + b), (w >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < BLK / 16; ++ks) {   // K of this product = the 128 columns j: 8 TMEM columns per step
+          // A: E of column half ks / 4 sits in the first 32 columns of that half of the S buffer;
           // B[K = j][N = l] is the Y tile itself read MN-major: 16 rows j per step = 2048 B
-          tc_mma_ts(tmG, tmE[b] + ks * 8, smem_desc_mn(sm0 + L::OFF_Y + st * L::Y_BYTES + ks * 2048, L::XB), ID2,
-                    (jb > 0 || ks > 0));
+          tc_mma_ts(tmG, tmS[b] + (ks / 4) * 64 + (ks % 4) * 8,
+                    smem_desc_mn(sm0 + L::OFF_Y + ys * L::Y_BYTES + ks * 2048, L::XB), ID2, (w > 0 || ks > 0));
         }
-        tc_commit(bar(B_EEMPTY + b));
-        tc_commit(bar(B_QEMPTY + st));
+        tc_commit(bar(L::B_YEMPTY + ys));
       }
-      if (ok) tc_commit(bar(B_GFULL));
+      if (ok) tc_commit(bar(L::B_GFULL));
     }
     __syncwarp();
   } else {
@@ -282,15 +288,32 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int row = q * 32 + lane;          // row inside the tile
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t rrow0 = sm0 + L::OFF_R + h * L::XB + row * 128;   // this row in the R tile (block h)
-    for (int jb = team; jb < NJ && ok; jb += 2) {
-      const int b = jb & 1, st = jb % NSTAGE;
-      ok = mbar_wait(bar(B_QFULL + st), (jb / NSTAGE) & 1);                   // R tile has landed
-      if (ok) ok = mbar_wait(bar(B_SFULL + b), (jb >> 1) & 1);                // S is complete
-      if (ok && jb >= 2) ok = mbar_wait(bar(B_EEMPTY + b), ((jb >> 1) - 1) & 1);  // E buffer is free again
+    if (team == 0) {
+      // the CTA's X block goes to TMEM once: lane = row, 32-bit column c = factor columns 2c, 2c + 1
+      const uint4 *xrow = reinterpret_cast<const uint4 *>(Xg + (size_t)(row0 + row) * K + h * (K / 2));
+#pragma unroll
+      for (int c = 0; c < K / 64; ++c) {
+        uint32_t xw[16];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const uint4 x4 = xrow[c * 4 + v];
+          xw[4 * v] = x4.x; xw[4 * v + 1] = x4.y; xw[4 * v + 2] = x4.z; xw[4 * v + 3] = x4.w;
+        }
+        tc_st16(tmX + lane_off + h * (K / 4) + c * 16, xw);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(L::B_XFULL));
+    }
+    for (int w = team; w < NW && ok; w += 2) {
+      const int b = w & 1, rs = w % L::NSR;
+      ok = mbar_wait(bar(L::B_RFULL + rs), (w / L::NSR) & 1);                 // R tile has landed
+      if (ok) ok = mbar_wait(bar(L::B_SFULL + b), (w >> 1) & 1);              // S is complete
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t rrow = rrow0 + st * L::R_BYTES;
+      const uint32_t rrow = rrow0 + rs * L::R_BYTES;
       uint32_t sv[2][32];
       tc_ld32_nowait(tmS[b] + lane_off + h * 64, sv[0]);
       tc_ld32_nowait(tmS[b] + lane_off + h * 64 + 32, sv[1]);
@@ -316,21 +339,22 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             ew[v * 4 + p] = *reinterpret_cast<uint32_t *>(&pk);
           }
         }
-        tc_st16(tmE[b] + lane_off + h * 32 + c2 * 16, ew);
+        // in place: this thread has already read all 64 S columns of its half
+        tc_st16(tmS[b] + lane_off + h * 64 + c2 * 16, ew);
       }
+      __syncwarp();   // every lane has its R values in registers: the stage can be refilled
+      if (lane == 0) mbar_arrive(bar(L::B_REMPTY + rs));
       tc_wait_st();
       // one arrival per warp: every lane orders its TMEM accesses, then lane 0 signals for the warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar(B_SEMPTY + b));
-        mbar_arrive(bar(B_EFULL + b));
-      }
+      if (lane == 0) mbar_arrive(bar(L::B_EFULL + b));
     }
-    if (ok && team == 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_GFULL), 0));
-    if (ok && team == 0) {
+    const bool writer = team == 0 && NW > 0;
+    if (ok && writer) ok = __all_sync(0xffffffffu, mbar_wait(bar(L::B_GFULL), 0));
+    if (ok && writer) {
       tc_fence_after();
-      float *grow = G + (size_t)(ib * BLK + row) * K + h * (K / 2);
+      float *grow = Gout + (size_t)(row0 + row) * K + h * (K / 2);
 #pragma unroll
       for (int c = 0; c < K / 64; ++c) {
         uint32_t gv[32];
@@ -347,6 +371,19 @@ dense_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// G[i] += part_0[i] + ... in this order (the partial blocks of the CTAs that shared a row block)
+__global__ void add_partials_kernel(float4 *__restrict__ G, const float4 *__restrict__ part, size_t n4, int nparts) {
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 g = G[i];
+    for (int p = 0; p < nparts; ++p) {
+      const float4 a = part[(size_t)p * n4 + i];
+      g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+    }
+    G[i] = g;
   }
 }
 
@@ -399,12 +436,29 @@ cudaError_t make_map(CUtensorMap *tm, CUtensorMapDataType dt, void *base, uint64
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// Number of CTAs per row block: fill the SMs when there are fewer row blocks than SMs, but leave every
+// CTA at least four column blocks.
+int dense_split(int rows_x, int rows_y) {
+  const int nrb = rows_x / BLK, nj = rows_y / BLK;
+  int sp = 148 / nrb;
+  if (sp > MAX_SPLIT) sp = MAX_SPLIT;
+  if (sp > nj / 4) sp = nj / 4;
+  return sp < 1 ? 1 : sp;
+}
+
 template <int K>
-cudaError_t launch_dense_pass(cudaStream_t st, const CUtensorMap &tmX, const CUtensorMap &tmY,
-                              const CUtensorMap &tmR, int rows_x, int rows_y, float *G, int32_t *flags) {
+cudaError_t launch_dense_pass(cudaStream_t st, const __nv_bfloat16 *X, const CUtensorMap &tmY,
+                              const CUtensorMap &tmR, int rows_x, int rows_y, float *G, float *Gpart,
+                              int32_t *flags) {
   auto kern = dense_pass_kernel<K>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<K>::TOTAL));
-  kern<<<rows_x / BLK, 576, Smem<K>::TOTAL, st>>>(tmX, tmY, tmR, rows_y, G, flags);
+  const int nrb = rows_x / BLK, nsplit = dense_split(rows_x, rows_y);
+  kern<<<nrb * nsplit, 576, Smem<K>::TOTAL, st>>>(X, tmY, tmR, rows_x, rows_y, nsplit, G, Gpart, flags);
+  if (nsplit > 1) {
+    const size_t n4 = (size_t)rows_x * K / 4;
+    add_partials_kernel<<<148 * 4, 256, 0, st>>>(reinterpret_cast<float4 *>(G), reinterpret_cast<const float4 *>(Gpart),
+                                                n4, nsplit - 1);
+  }
   return cudaGetLastError();
 }
 
@@ -419,7 +473,8 @@ void dense_carve(tsid_template *t, const tsid_config_t &c, Carver &cv) {
   DenseState *d = t->dense;
   const size_t mn = (size_t)c.m * c.n;
   __half *R = cv.take<__half>(mn), *RT = cv.take<__half>(mn);
-  if (d) { d->R = R; d->RT = RT; }
+  float *gpart = cv.take<float>((size_t)(MAX_SPLIT - 1) * (c.m > c.n ? c.m : c.n) * c.k);
+  if (d) { d->R = R; d->RT = RT; d->gpart = gpart; }
 }
 
 DenseState *dense_new() { return new (std::nothrow) DenseState; }
@@ -445,20 +500,26 @@ cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag) {
   return cudaSuccess;
 }
 
+// two passes + the update kernels of the two sides, + one add per pass whose column range is split
+int dense_launches_per_step(const tsid_template *t) {
+  const tsid_config_t &c = t->cfg;
+  return 4 + (dense_split(c.m, c.n) > 1) + (dense_split(c.n, c.m) > 1);
+}
+
 // G_P and G_Q from the current bf16 shadows (which must be up to date).
 cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ) {
   DenseState *d = t->dense;
   const tsid_config_t &c = t->cfg;
   cudaStream_t st = t->stream;
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW0], st);
-  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmP, d->tmQ, d->tmR, c.m, c.n, GP, t->flags));
-  else CK(launch_dense_pass<64>(st, d->tmP, d->tmQ, d->tmR, c.m, c.n, GP, t->flags));
+  if (c.k == 128) CK(launch_dense_pass<128>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags));
+  else CK(launch_dense_pass<64>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags));
   if (t->prof.on && t->prof.nsteps < kProfSteps) {
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW1], st);
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL0], st);
   }
-  if (c.k == 128) CK(launch_dense_pass<128>(st, d->tmQ, d->tmP, d->tmRT, c.n, c.m, GQ, t->flags));
-  else CK(launch_dense_pass<64>(st, d->tmQ, d->tmP, d->tmRT, c.n, c.m, GQ, t->flags));
+  if (c.k == 128) CK(launch_dense_pass<128>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags));
+  else CK(launch_dense_pass<64>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags));
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL1], st);
   return cudaSuccess;
 }

@@ -138,6 +138,7 @@ DenseState *dense_new();
 void dense_delete(DenseState *d);
 void dense_carve(tsid_template *t, const tsid_config_t &c, Carver &cv);
 cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag);
+int dense_launches_per_step(const tsid_template *t);
 cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ);
 
 inline int bits_for(uint32_t maxval) {  // number of bits needed to represent values <= maxval
