@@ -25,10 +25,13 @@ def _bernoulli(m, n, k, density, seed, **kw):
                       seed=seed, **base)
 
 
-@pytest.mark.parametrize("m,n,k", [(256, 128, 64), (128, 384, 128), (512, 256, 128)])
+@pytest.mark.parametrize("m,n,k", [(256, 128, 64), (128, 384, 128), (512, 256, 128), (256, 2048, 64),
+                                   (19200, 512, 64)])
 def test_dense_exact_on_small_integers(m, n, k):
     """Integer factors and ratings: every product, residual and sum is exact in bf16/fp16/fp32, so the
-    tensor-core path must reproduce the oracle bit for bit (any wrong tile, swizzle or descriptor shows)."""
+    tensor-core path must reproduce the oracle bit for bit (any wrong tile, swizzle or descriptor shows).
+    256 x 2048 makes several CTAs share a row block (column range split, partial gradient blocks added
+    in a fixed order); 19200 x 512 has more row blocks than SMs in one pass and a split in the other."""
     rng = np.random.default_rng(m + n + k)
     P = rng.integers(-2, 3, (m, k)).astype(np.float32); Q = rng.integers(-2, 3, (n, k)).astype(np.float32)
     mask = rng.random((m, n)) < 0.3
