@@ -47,6 +47,18 @@ def test_layout_shapes(m, n, nnz, pos):
     _check(m, n, r, c, v)
 
 
+@pytest.mark.parametrize("m,n", [(20_000_000, 130), (130, 20_000_000), (17_000_000, 17_000_000)])
+def test_layout_four_pass_sorts(m, n):
+    """More than 2^24 rows or columns: four radix passes per sort, so the sorts end in the other buffer set
+    than with the three passes of the workload sizes."""
+    rng = np.random.default_rng(m % 1000 + n % 1000)
+    nnz = 120_000
+    key = np.unique(rng.integers(0, m, nnz).astype(np.int64) * n + rng.integers(0, n, nnz))
+    key = key[rng.permutation(len(key))]
+    rows, cols = (key // n).astype(np.int32), (key % n).astype(np.int32)
+    _check(m, n, rows, cols, rng.standard_normal(len(key)).astype(np.float32), k=4)
+
+
 def test_layout_degenerate_cases():
     _check(7, 5, np.zeros(0, np.int32), np.zeros(0, np.int32), np.zeros(0, np.float32))     # empty Omega
     _check(7, 5, np.array([3], np.int32), np.array([4], np.int32), np.array([2.5], np.float32))
