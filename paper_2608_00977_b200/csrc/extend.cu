@@ -25,8 +25,11 @@ namespace {
   } while (0)
 
 // Register-tiled fp32 GEMM: BM x BN output tile per 256-thread block, 8 x 8 outputs per thread (two 4-wide
-// halves in each direction so that shared-memory reads are conflict-free float4s), BK-deep slices.
-// A is [M][K] row-major.  B is [K][N] row-major, or with B_NK = true [N][K] row-major.
+// halves in each direction so that shared-memory reads are conflict-free float4s), BK-deep slices, two
+// shared-memory buffers: the next slice travels global -> registers while the current one is multiplied.
+// A is [M][K] row-major.  B is [K][N] row-major, or with B_NK = true [N][K] row-major.  VEC = every row
+// of A, B and of the epilogue's matrices starts 16-byte aligned and K, N are multiples of 4 (then global
+// memory is read and written as float4).
 constexpr int BM = 128, BK = 16;   // BN (128 or 64) is a template parameter
 constexpr int kSplitW = 8;         // K-splits of the tall-skinny first GEMM (K = d is long, M x N is small)
 
@@ -40,76 +43,161 @@ struct SplitEpi {       // partial[z][m][n] = acc   (z = K-split index; summed i
   __device__ __forceinline__ void operator()(int gm, int gn, int N, float acc) const {
     part[blockIdx.z * plane + (size_t)gm * N + gn] = acc;
   }
+  __device__ __forceinline__ void vec4(int gm, int gn, int N, float4 acc) const {
+    *reinterpret_cast<float4 *>(part + blockIdx.z * plane + (size_t)gm * N + gn) = acc;
+  }
+  __device__ __forceinline__ void prefetch(int, int, int) const {}
 };
 struct AdamEpi {        // g = -2 acc + 2 lambda C; Adam update of C and its moments in place
   float *Cm, *Mo, *Vo;
   AdamArgs a;
+  __device__ __forceinline__ float one(float acc, float c, float &mo, float &vo) const {
+    const float g = fmaf(a.lam2, c, -2.f * acc);
+    mo = fmaf(a.b1, mo, (1.f - a.b1) * g);
+    vo = fmaf(a.b2, vo, (1.f - a.b2) * g * g);
+    // (the quotient uses the fast reciprocal: 2 ulp on a step that is itself ~lr in size)
+    return c - __fdividef(a.lr * (mo * a.c1), sqrtf(vo * a.c2) + a.eps);
+  }
   __device__ __forceinline__ void operator()(int gm, int gn, int N, float acc) const {
     const size_t o = (size_t)gm * N + gn;
-    const float c = Cm[o];
-    const float g = fmaf(a.lam2, c, -2.f * acc);
-    const float mo = fmaf(a.b1, Mo[o], (1.f - a.b1) * g);
-    const float vo = fmaf(a.b2, Vo[o], (1.f - a.b2) * g * g);
+    float mo = Mo[o], vo = Vo[o];
+    Cm[o] = one(acc, Cm[o], mo, vo);
     Mo[o] = mo;
     Vo[o] = vo;
-    Cm[o] = c - a.lr * (mo * a.c1) / (sqrtf(vo * a.c2) + a.eps);
+  }
+  __device__ __forceinline__ void vec4(int gm, int gn, int N, float4 acc) const {
+    const size_t o = (size_t)gm * N + gn;
+    float4 c = *reinterpret_cast<const float4 *>(Cm + o), mo = *reinterpret_cast<const float4 *>(Mo + o),
+           vo = *reinterpret_cast<const float4 *>(Vo + o);
+    c.x = one(acc.x, c.x, mo.x, vo.x);
+    c.y = one(acc.y, c.y, mo.y, vo.y);
+    c.z = one(acc.z, c.z, mo.z, vo.z);
+    c.w = one(acc.w, c.w, mo.w, vo.w);
+    *reinterpret_cast<float4 *>(Cm + o) = c;
+    *reinterpret_cast<float4 *>(Mo + o) = mo;
+    *reinterpret_cast<float4 *>(Vo + o) = vo;
+  }
+  // asks L2 for the three 16-byte pieces this thread will update, so that they arrive during the main loop
+  __device__ __forceinline__ void prefetch(int gm, int gn, int N) const {
+    const size_t o = (size_t)gm * N + gn;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(Cm + o));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(Mo + o));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(Vo + o));
   }
 };
 
-template <int BN, bool B_NK, class Epi>
+// four consecutive elements of row `row` of a row-major matrix with leading dimension ld, zero outside
+// [0, nrows) x [0, colend)
+template <bool VEC>
+__device__ __forceinline__ float4 fetch4(const float *__restrict__ P, int row, int col, int nrows, int ld, int colend) {
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (row < nrows) {
+    const float *src = P + (size_t)row * ld + col;
+    if (VEC) {
+      if (col < colend) v = __ldg(reinterpret_cast<const float4 *>(src));
+    } else {
+      if (col < colend) v.x = __ldg(src);
+      if (col + 1 < colend) v.y = __ldg(src + 1);
+      if (col + 2 < colend) v.z = __ldg(src + 2);
+      if (col + 3 < colend) v.w = __ldg(src + 3);
+    }
+  }
+  return v;
+}
+
+template <int BN, bool B_NK, bool VEC, class Epi>
 __global__ void __launch_bounds__(256)
 gemm_kernel(const float *__restrict__ A, const float *__restrict__ B, int M, int N, int K, int kper, Epi epi) {
   constexpr int TH = BN / 32;   // half of the thread's columns: 4 (BN = 128) or 2 (BN = 64)
-  __shared__ __align__(16) float As[BK][BM], Bs[BK][BN];
+  constexpr int NA = BM * BK / 4 / 256, NB = BN * BK / 4 / 256;   // float4 loads per thread and slice
+  __shared__ __align__(16) float As[2][BK][BM], Bs[2][BK][BN];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
   const int kbeg = blockIdx.z * kper, kend = kbeg + kper < K ? kbeg + kper : K;
   float acc[8][2 * TH] = {};
-  for (int k0 = kbeg; k0 < kend; k0 += BK) {
+  float4 ra[NA], rb[NB];
+  auto load_slice = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < (BM * BK) / 256; ++i) {
+    for (int i = 0; i < NA; ++i) {   // lanes run along the rows, so the transposed store below is conflict-free
       const int q = threadIdx.x + i * 256;
-      const int r = q / BK, c = q % BK;
-      const int gm = m0 + r, gk = k0 + c;
-      As[c][r] = (gm < M && gk < kend) ? __ldg(A + (size_t)gm * K + gk) : 0.f;
+      ra[i] = fetch4<VEC>(A, m0 + q % BM, k0 + (q / BM) * 4, M, K, kend);
     }
 #pragma unroll
-    for (int i = 0; i < (BN * BK) / 256; ++i) {
+    for (int i = 0; i < NB; ++i) {
+      const int q = threadIdx.x + i * 256;
+      if (B_NK) rb[i] = fetch4<VEC>(B, n0 + q % BN, k0 + (q / BN) * 4, N, K, kend);
+      else rb[i] = fetch4<VEC>(B, k0 + q / (BN / 4), n0 + (q % (BN / 4)) * 4, kend, N, N);
+    }
+  };
+  auto store_slice = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < NA; ++i) {
+      const int q = threadIdx.x + i * 256, r = q % BM, c = (q / BM) * 4;
+      As[buf][c][r] = ra[i].x; As[buf][c + 1][r] = ra[i].y; As[buf][c + 2][r] = ra[i].z; As[buf][c + 3][r] = ra[i].w;
+    }
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
       const int q = threadIdx.x + i * 256;
       if (B_NK) {
-        const int r = q / BK, c = q % BK;
-        const int gn = n0 + r, gk = k0 + c;
-        Bs[c][r] = (gn < N && gk < kend) ? __ldg(B + (size_t)gn * K + gk) : 0.f;
+        const int r = q % BN, c = (q / BN) * 4;
+        Bs[buf][c][r] = rb[i].x; Bs[buf][c + 1][r] = rb[i].y; Bs[buf][c + 2][r] = rb[i].z; Bs[buf][c + 3][r] = rb[i].w;
       } else {
-        const int rb = q / BN, cb = q % BN;
-        const int gkb = k0 + rb, gn = n0 + cb;
-        Bs[rb][cb] = (gkb < kend && gn < N) ? __ldg(B + (size_t)gkb * N + gn) : 0.f;
+        *reinterpret_cast<float4 *>(&Bs[buf][q / (BN / 4)][(q % (BN / 4)) * 4]) = rb[i];
       }
     }
-    __syncthreads();
+  };
+  if (kbeg < kend) {
+    load_slice(kbeg);
+    store_slice(0);
+  }
+  if (VEC && TH == 4) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int gm = m0 + (i < 4 ? ty * 4 + i : BM / 2 + ty * 4 + i - 4);
+#pragma unroll
+      for (int hcol = 0; hcol < 2; ++hcol) {
+        const int gn = n0 + hcol * (BN / 2) + tx * 4;
+        if (gm < M && gn < N) epi.prefetch(gm, gn, N);
+      }
+    }
+  }
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = kbeg; k0 < kend; k0 += BK, buf ^= 1) {
+    const bool more = k0 + BK < kend;
+    if (more) load_slice(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      const float4 a0 = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
-      const float4 a1 = *reinterpret_cast<const float4 *>(&As[kk][BM / 2 + ty * 4]);
+      const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][kk][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][kk][BM / 2 + ty * 4]);
       const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
       float b[2 * TH];
 #pragma unroll
-      for (int j = 0; j < TH; ++j) { b[j] = Bs[kk][tx * TH + j]; b[TH + j] = Bs[kk][BN / 2 + tx * TH + j]; }
+      for (int j = 0; j < TH; ++j) { b[j] = Bs[buf][kk][tx * TH + j]; b[TH + j] = Bs[buf][kk][BN / 2 + tx * TH + j]; }
 #pragma unroll
       for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 2 * TH; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
+    if (more) store_slice(buf ^ 1);   // the other buffer was last read before the previous barrier
     __syncthreads();
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int gm = m0 + (i < 4 ? ty * 4 + i : BM / 2 + ty * 4 + i - 4);
     if (gm >= M) continue;
+    if (VEC && TH == 4) {
 #pragma unroll
-    for (int j = 0; j < 2 * TH; ++j) {
-      const int gn = n0 + (j < TH ? tx * TH + j : BN / 2 + tx * TH + j - TH);
-      if (gn < N) epi(gm, gn, N, acc[i][j]);
+      for (int hcol = 0; hcol < 2; ++hcol) {
+        const int gn = n0 + hcol * (BN / 2) + tx * 4;
+        if (gn < N) epi.vec4(gm, gn, N, make_float4(acc[i][hcol * 4], acc[i][hcol * 4 + 1], acc[i][hcol * 4 + 2], acc[i][hcol * 4 + 3]));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 2 * TH; ++j) {
+        const int gn = n0 + (j < TH ? tx * TH + j : BN / 2 + tx * TH + j - TH);
+        if (gn < N) epi(gm, gn, N, acc[i][j]);
+      }
     }
   }
 }
@@ -301,8 +389,13 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
     const int nsplit = (d + kper - 1) / kper;
     const dim3 gw((nc + BM - 1) / BM, (k + 63) / 64, nsplit), ga((nc + BM - 1) / BM, (d + 127) / 128, 1);
     const size_t plane = (size_t)nc * k;
+    // float4 paths need every matrix row 16-byte aligned: k is a multiple of 4 by contract, d need not be
+    const bool vec = d % 4 == 0 && k % 4 == 0 && ((reinterpret_cast<uintptr_t>(sl.CT) | reinterpret_cast<uintptr_t>(d_Q) |
+                                                  reinterpret_cast<uintptr_t>(e.U) | reinterpret_cast<uintptr_t>(e.Mo) |
+                                                  reinterpret_cast<uintptr_t>(e.Vo) | reinterpret_cast<uintptr_t>(e.Wpart)) & 15u) == 0;
     auto gemm_w = [&]() {
-      gemm_kernel<64, false, SplitEpi><<<gw, 256, 0, s_cmp>>>(sl.CT, d_Q, nc, k, d, kper, SplitEpi{e.Wpart, plane});
+      if (vec) gemm_kernel<64, false, true, SplitEpi><<<gw, 256, 0, s_cmp>>>(sl.CT, d_Q, nc, k, d, kper, SplitEpi{e.Wpart, plane});
+      else gemm_kernel<64, false, false, SplitEpi><<<gw, 256, 0, s_cmp>>>(sl.CT, d_Q, nc, k, d, kper, SplitEpi{e.Wpart, plane});
       sum_splits_kernel<<<148 * 2, 256, 0, s_cmp>>>(e.Wpart, plane, nsplit, e.W);
     };
     double p1 = 1.0, p2 = 1.0;
@@ -312,7 +405,8 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
       p1 *= cfg->beta1; p2 *= cfg->beta2;
       AdamArgs aa{cfg->eta, 2.f * cfg->lambda, cfg->beta1, cfg->beta2, cfg->eps, (float)(1.0 / (1.0 - p1)),
                   (float)(1.0 / (1.0 - p2))};
-      gemm_kernel<128, true, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
+      if (vec) gemm_kernel<128, true, true, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
+      else gemm_kernel<128, true, false, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
     }
     if (h_sse_or_null) {
       gemm_w();
