@@ -318,6 +318,53 @@ def measure_extend(args, w, tpl, B, dev):
                                    "fp32_tflops": flops / t / 1e12}}))
 
 
+def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
+    """One template sharded by rows over the ranks: per step tsid_grad, one all-reduce (sum) of G_Q over
+    NCCL, tsid_apply.  Total work is fixed as the rank count grows."""
+    from paper_2608_00977_b200 import sharded as S
+    r0, r1 = S.row_block(w.m, rank, world)
+    rows, cols, vals = S.shard_coo(tpl.rows, tpl.cols, tpl.vals, r0, r1)
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    sh = S.RowShard(r1 - r0, w.n, w.k, rows, cols, vals, precision=prec, eta=w.eta, lam=w.lam, xi=w.xi, clip=w.clip,
+                    norm_p=w.norm_p, norm_q=w.norm_q, dist=dist)
+    P, Q = tpl.P0[r0:r1].clone().contiguous(), tpl.Q0.clone()
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+    for _ in range(args.warmup):
+        sh.step(P, Q)
+    sh.T.tsid_check()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        sh.step(P, Q)
+    b.record(stream)
+    barrier()
+    ms = max_over_ranks(a.elapsed_time(b), dist, dev)
+    clocks = sampler.stop()
+    sh.T.tsid_check()
+    sse = sh.sse(P, Q)
+    if rank == 0:
+        _, launches = sh.T.tsid_get_info()
+        print(json.dumps({"metric": METRIC, "value": tpl.nnz * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+                          "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                          "dtype": "bf16" if w.precision == "bf16" else "f32", "data": "synthetic",
+                          "config": {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": tpl.nnz,
+                                     "parallelism": "rows/%d, all-reduce(sum) of G_Q (%d bytes) per step" % (world, w.n * w.k * 4),
+                                     "l2": "inputs larger than L2, steps timed back to back"},
+                          "clocks": clocks, "e2e": None, "gpu_launches": launches * args.steps, "roofline": None,
+                          "cpu_baseline": None, "rmse_after": (sse / tpl.nnz) ** 0.5}))
+    sh.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -333,6 +380,9 @@ def main():
                          "layout: the layout pass (tsid_template_create) on the workload's COO in --order")
     ap.add_argument("--order", default="shuffled", choices=["sorted", "shuffled"],
                     help="entry order of the COO input for --measure layout")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
+                    help="N > 1: independent replicas of the template (default), or ONE template sharded by rows "
+                         "with one all-reduce of G_Q per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -377,6 +427,9 @@ def main():
         return
     if args.measure == "layout":
         measure_layout(args, w, tpl, B, dev)
+        return
+    if args.shard == "rows":
+        run_row_sharded(args, w, tpl, B, dev, dist, rank, world)
         return
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
     want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]

@@ -134,6 +134,28 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
 tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *d_gradP_or_null,
                              float *d_gradQ_or_null);
 
+/* The two halves of tsid_grad_step, for a template whose rows are sharded over several GPUs
+ * (the paper keeps template recovery on one GPU and names multi-GPU recovery as future work,
+ * Sec. 7; the full-batch step itself splits exactly: with the rows of Omega partitioned over the
+ * ranks, each rank's G_P rows are complete and the G_Q of all ranks add up, so one sum-exchange of
+ * G_Q per step is the only communication).
+ *   tsid_grad: the raw sums G_P = E Q (m x k) and G_Q = E^T P (n x k) of THIS template's entries
+ *     at (d_P, d_Q); nothing is updated.  With TSID_CLIP_ASYM_ENTRY the sums are those of the
+ *     clipped per-entry directions, which add up over shards in the same way.
+ *   tsid_apply: direction, clip and update of tsid_grad_step from given sums (for example d_GQ
+ *     summed over the ranks), in place on d_P, d_Q; refreshes the bf16 shadows.
+ *   tsid_get_counts: |Omega_i| (int32[m]) and |Omega^j| (int32[n]) of this template; either may be NULL.
+ *   tsid_set_norm_counts: replaces the counts that TSID_NORM_COUNT divides by (a shard sees only
+ *     its part of every column: pass the counts summed over the ranks); NULL leaves a side as it is.
+ *     Lasts until destroy.
+ * All four are asynchronous on cfg.stream; every pointer is a 16-byte aligned DEVICE pointer.
+ * Errors: TSID_ERR_INVALID_ARG. */
+tsid_status_t tsid_grad(tsid_template_t *t, const float *d_P, const float *d_Q, float *d_GP, float *d_GQ);
+tsid_status_t tsid_apply(tsid_template_t *t, float *d_P, float *d_Q, const float *d_GP, const float *d_GQ);
+tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int32_t *d_cnt_q_or_null);
+tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or_null,
+                                   const int32_t *d_cnt_q_or_null);
+
 /* `epochs` steps in place.  loss_every > 0: after every loss_every-th step (and before the
  * first) the SSE is computed and stored in h_sse_history_or_null (host, capacity
  * 1 + epochs / loss_every doubles); this synchronises.  loss_every == 0: asynchronous. */

@@ -32,7 +32,8 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_check", "tsid_destroy", "tsid_get_layout", "tsid_residuals", "tsid_get_info",
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
-           "tsid_extend_workspace_bytes", "tsid_extend"]
+           "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
+           "tsid_set_norm_counts"]
 
 
 class TsidConfig(C.Structure):
@@ -74,6 +75,10 @@ def lib():
         L.tsid_template_create.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, C.POINTER(vp)]
         L.tsid_grad_step.argtypes = [vp, vp, vp, vp, vp]
         L.tsid_fit.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.tsid_grad.argtypes = [vp, vp, vp, vp, vp]
+        L.tsid_apply.argtypes = [vp, vp, vp, vp, vp]
+        L.tsid_get_counts.argtypes = [vp, vp, vp]
+        L.tsid_set_norm_counts.argtypes = [vp, vp, vp]
         L.tsid_loss.argtypes = [vp, vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.tsid_check.argtypes = [vp]
         L.tsid_destroy.argtypes = [vp]
@@ -164,6 +169,40 @@ class Template:
         st = lib().tsid_grad_step(self.h, P.data_ptr(), Q.data_ptr(),
                                   gradP.data_ptr() if gradP is not None else None,
                                   gradQ.data_ptr() if gradQ is not None else None)
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_grad(self, P, Q, gradP, gradQ):
+        self._factors(P, Q)
+        _check_tensor(gradP, torch.float32, self.m * self.k, "gradP")
+        _check_tensor(gradQ, torch.float32, self.n * self.k, "gradQ")
+        st = lib().tsid_grad(self.h, P.data_ptr(), Q.data_ptr(), gradP.data_ptr(), gradQ.data_ptr())
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_apply(self, P, Q, gradP, gradQ):
+        self._factors(P, Q)
+        _check_tensor(gradP, torch.float32, self.m * self.k, "gradP")
+        _check_tensor(gradQ, torch.float32, self.n * self.k, "gradQ")
+        st = lib().tsid_apply(self.h, P.data_ptr(), Q.data_ptr(), gradP.data_ptr(), gradQ.data_ptr())
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_get_counts(self):
+        cp = torch.empty(self.m, dtype=torch.int32, device=self.device)
+        cq = torch.empty(self.n, dtype=torch.int32, device=self.device)
+        st = lib().tsid_get_counts(self.h, cp.data_ptr(), cq.data_ptr())
+        if st != TSID_OK:
+            self._raise(st)
+        return cp, cq
+
+    def tsid_set_norm_counts(self, cnt_p=None, cnt_q=None):
+        if cnt_p is not None:
+            _check_tensor(cnt_p, torch.int32, self.m, "cnt_p")
+        if cnt_q is not None:
+            _check_tensor(cnt_q, torch.int32, self.n, "cnt_q")
+        st = lib().tsid_set_norm_counts(self.h, cnt_p.data_ptr() if cnt_p is not None else None,
+                                        cnt_q.data_ptr() if cnt_q is not None else None)
         if st != TSID_OK:
             self._raise(st)
 

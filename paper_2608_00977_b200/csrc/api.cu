@@ -188,6 +188,41 @@ tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *
   return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
 }
 
+tsid_status_t tsid_grad(tsid_template_t *t, const float *d_P, const float *d_Q, float *d_GP, float *d_GQ) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  if (!d_GP || !d_GQ || !aligned16(d_GP) || !aligned16(d_GQ))
+    return fail(t, TSID_ERR_INVALID_ARG, "gradient outputs must be non-null and 16-byte aligned");
+  cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
+  if (e == cudaSuccess) e = grad_any(t, d_P, d_Q, d_GP, d_GQ);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+tsid_status_t tsid_apply(tsid_template_t *t, float *d_P, float *d_Q, const float *d_GP, const float *d_GQ) {
+  tsid_status_t st = check_factors(t, d_P, d_Q);
+  if (st != TSID_OK) return st;
+  if (!d_GP || !d_GQ || !aligned16(d_GP) || !aligned16(d_GQ))
+    return fail(t, TSID_ERR_INVALID_ARG, "gradient inputs must be non-null and 16-byte aligned");
+  cudaError_t e = sparse_update(t, d_P, d_Q, d_GP, d_GQ);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int32_t *d_cnt_q_or_null) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  cudaError_t e = cudaSuccess;
+  if (d_cnt_p_or_null) e = sparse_counts(t, t->rowside, d_cnt_p_or_null);
+  if (e == cudaSuccess && d_cnt_q_or_null) e = sparse_counts(t, t->colside, d_cnt_q_or_null);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
+tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or_null, const int32_t *d_cnt_q_or_null) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  cudaError_t e = cudaSuccess;
+  if (d_cnt_p_or_null) e = sparse_scale_from_counts(t, t->rowside, t->cfg.norm_p, d_cnt_p_or_null);
+  if (e == cudaSuccess && d_cnt_q_or_null) e = sparse_scale_from_counts(t, t->colside, t->cfg.norm_q, d_cnt_q_or_null);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
 static tsid_status_t loss_sync(tsid_template *t, const float *d_P, const float *d_Q, double *sse, double *sq) {
   cudaError_t e = sparse_loss(t, d_P, d_Q, t->red);
   double h[2] = {0, 0};

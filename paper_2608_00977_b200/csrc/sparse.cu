@@ -459,6 +459,27 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
   return cudaGetLastError();
 }
 
+__global__ void counts_kernel(const int64_t *__restrict__ ptr, int32_t nrows, int32_t *__restrict__ cnt) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nrows; i += (int64_t)gridDim.x * blockDim.x)
+    cnt[i] = (int32_t)(ptr[i + 1] - ptr[i]);
+}
+// scale = 2 / s with s = max(1, count) under NORM_COUNT, 1 otherwise (the same rule as at create)
+__global__ void scale_kernel(const int32_t *__restrict__ cnt, int32_t nrows, int norm_count, float *__restrict__ scale) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nrows; i += (int64_t)gridDim.x * blockDim.x) {
+    const int32_t c = cnt[i];
+    scale[i] = 2.0f / ((norm_count && c > 1) ? (float)c : 1.0f);
+  }
+}
+
+cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt) {
+  counts_kernel<<<ew_grid(sd.nrows), 256, 0, t->stream>>>(sd.ptr, sd.nrows, d_cnt);
+  return cudaGetLastError();
+}
+cudaError_t sparse_scale_from_counts(tsid_template *t, Side &sd, int norm_mode, const int32_t *d_cnt) {
+  scale_kernel<<<ew_grid(sd.nrows), 256, 0, t->stream>>>(d_cnt, sd.nrows, norm_mode == TSID_NORM_COUNT, sd.scale);
+  return cudaGetLastError();
+}
+
 cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_Q, float *d_e) {
   const bool bf = t->cfg.precision == TSID_BF16_SHADOW;
   CK(sparse_convert_shadow(t, d_P, d_Q));

@@ -128,6 +128,8 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
 cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_Q, float *d_e);
 cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
 int sparse_launches_per_step(const tsid_template *t);
+cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt);
+cudaError_t sparse_scale_from_counts(tsid_template *t, Side &sd, int norm_mode, const int32_t *d_cnt);
 cudaError_t sparse_side_grad(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G);
 cudaError_t sparse_side_sse(tsid_template *t, const Side &sd, const void *stage, const void *gather, double *red,
                             double *d_out);

@@ -1,0 +1,88 @@
+"""Row-sharded template recovery (tsid_grad, one sum of G_Q, tsid_apply) against the oracle's full-batch
+steps.  One GPU is enough: the shards of a template run one after the other and their G_Q buffers are
+summed here, which is all an all-reduce does."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import F32_TOL, np_coo, relerr, small_workload
+from paper_2608_00977_b200 import binding as B
+from paper_2608_00977_b200 import sharded as S
+from paper_2608_00977_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+CASES = {
+    "plain": dict(precision="f32", eta=0.01, lam=0.0, clip=W.CLIP_NONE, norm_p=W.NORM_NONE, norm_q=W.NORM_NONE),
+    "clip-count": dict(precision="f32", eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT,
+                       norm_q=W.NORM_COUNT),
+    "paper-literal": dict(precision="f32", eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_ENTRY, norm_p=W.NORM_NONE,
+                          norm_q=W.NORM_COUNT),
+    "bf16": dict(precision="bf16", eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT,
+                 norm_q=W.NORM_COUNT),
+}
+
+
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_steps_match_the_full_batch_oracle(case, world):
+    kw = CASES[case]
+    m, n, k, nnz, steps = 1501, 700, 32, 120_000, 3
+    w = small_workload("shard-" + case, m, n, k, nnz, positions="zipf", seed=11 + world, **kw)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    shards, Ps, Qs = [], [], []
+    for r in range(world):
+        r0, r1 = S.row_block(m, r, world)
+        rows, cols, vals = S.shard_coo(tpl.rows, tpl.cols, tpl.vals, r0, r1)
+        shards.append(S.RowShard(r1 - r0, n, k, rows, cols, vals, precision=prec, eta=w.eta, lam=w.lam, xi=w.xi,
+                                 clip=w.clip, norm_p=w.norm_p, norm_q=w.norm_q))
+        Ps.append(tpl.P0[r0:r1].clone().contiguous())
+        Qs.append(tpl.Q0.clone())
+    # the exchange of the column counts, then of G_Q in every step
+    cq = sum(s.col_counts.clone() for s in shards)
+    assert int(cq.sum()) == tpl.nnz
+    for s in shards:
+        s.set_global_col_counts(cq)
+    for _ in range(steps):
+        for s, P, Q in zip(shards, Ps, Qs):
+            s.grad(P.view(-1), Q.view(-1))
+        total = shards[0].GQ.clone()
+        for s in shards[1:]:
+            total += s.GQ
+        for s, P, Q in zip(shards, Ps, Qs):
+            s.GQ.copy_(total)
+            s.apply(P.view(-1), Q.view(-1))
+            s.T.tsid_check()
+    for Q in Qs[1:]:
+        assert torch.equal(Q, Qs[0])                      # the replicas never drift apart
+    rows, cols, vals = np_coo(tpl)
+    bf = w.precision == "bf16"
+    Pr, Qr, _ = oracle.fit(m, n, k, rows, cols, vals, tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy(), steps, w.eta, w.lam,
+                           w.xi, w.clip, w.norm_p, w.norm_q, bf16_emulate=bf, history=False)
+    tol = 2e-3 if bf else F32_TOL      # bf16: the shadows of later steps round slightly different fp32 values
+    assert relerr(torch.cat(Ps).cpu().numpy(), Pr) <= tol
+    assert relerr(Qs[0].cpu().numpy(), Qr) <= tol
+    # the global SSE is the sum of the shards' SSEs
+    sse = sum(s.T.tsid_loss(P.view(-1), Q.view(-1))[0] for s, P, Q in zip(shards, Ps, Qs))
+    ref_sse, _ = oracle.loss(m, n, k, rows, cols, vals, Pr, Qr, w.lam, bf16_emulate=bf)
+    assert abs(sse - ref_sse) <= (2e-2 if bf else 1e-4) * ref_sse
+    for s in shards:
+        s.destroy()
+
+
+def test_one_shard_equals_grad_step_bitwise():
+    w = small_workload("shard-one", 900, 400, 16, 40_000, seed=5, eta=0.05, lam=0.03, clip=W.CLIP_ASYM_STEP,
+                       norm_p=W.NORM_COUNT, norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV)
+    s = S.RowShard(w.m, w.n, w.k, tpl.rows, tpl.cols, tpl.vals, eta=w.eta, lam=w.lam, xi=w.xi, clip=w.clip,
+                   norm_p=w.norm_p, norm_q=w.norm_q)
+    T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    Pa, Qa, Pb, Qb = tpl.P0.clone(), tpl.Q0.clone(), tpl.P0.clone(), tpl.Q0.clone()
+    for _ in range(3):
+        s.step(Pa.view(-1), Qa.view(-1))
+        T.tsid_grad_step(Pb.view(-1), Qb.view(-1))
+    assert torch.equal(Pa, Pb) and torch.equal(Qa, Qb)
+    s.destroy(); T.tsid_destroy()
