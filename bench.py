@@ -112,15 +112,15 @@ def aggregate_value(world, units_per_rank_step, steps, seconds):
     return world * units_per_rank_step * steps / seconds
 
 
-def alg_bytes(w, nnz, nseg_row, nseg_col):
+def alg_bytes(w, nnz, nseg_row, nseg_col, value_bytes=4):
     """Algorithmic bytes of one launch of each kernel of a step.  A pass reads per entry a 4-byte index, a
     4-byte value and one gathered factor row (k*b bytes, b = 2 for bf16 shadows, 4 for fp32), and per row the
     staged factor row (k*b), a 16-byte segment descriptor, and writes the gradient row (4k).  The update reads
     gradient and master, writes master (and the bf16 shadow), and reads one scale per row."""
     b = 2 if w.precision == "bf16" else 4
     k = w.k
-    row = nnz * (8 + k * b) + w.m * k * (b + 4) + nseg_row * 16
-    col = nnz * (8 + k * b) + w.n * k * (b + 4) + nseg_col * 16
+    row = nnz * (4 + value_bytes + k * b) + w.m * k * (b + 4) + nseg_row * 16
+    col = nnz * (4 + value_bytes + k * b) + w.n * k * (b + 4) + nseg_col * 16
     upd = (w.m + w.n) * k * (4 + 4 + 4 + (b if b == 2 else 0)) + (w.m + w.n) * 4
     return row, col, upd
 
@@ -383,6 +383,8 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
                     help="N > 1: independent replicas of the template (default), or ONE template sharded by rows "
                          "with one all-reduce of G_Q per step")
+    ap.add_argument("--values", default="f32", choices=["f32", "u8"],
+                    help="u8: stream the ratings as one byte each (TSID_VALUES_U8; needs integer values, e.g. C2, C3, C5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
@@ -433,7 +435,8 @@ def main():
         return
     prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
     want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]
-    T = B.template_from_workload(tpl, path=want_path)
+    vflags = B.TSID_VALUES_U8 if args.values == "u8" else 0
+    T = B.template_from_workload(tpl, path=want_path, flags=vflags)
     torch.cuda.synchronize(dev)
     if rank == 0:
         sys.stderr.write("[bench] %s: generated %d entries in %.1f s, layout pass %.2f s, workspace %.2f GB\n" % (
@@ -495,7 +498,7 @@ def main():
     peak, tf_sustained, tf_burst, peak_kind = load_peaks()
     nseg_row = w.m + nnz // 1024
     nseg_col = w.n + nnz // 1024
-    b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col)
+    b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col, 1 if args.values == "u8" else 4)
     pass_ms = (row_ms + col_ms) / max(1, 2 * nrec)
     bytes_per_launch = (b_row + b_col) / 2
     achieved = bytes_per_launch / (pass_ms * 1e-3) / 1e9 if pass_ms > 0 else 0.0
@@ -578,6 +581,7 @@ def main():
                 "config": {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": nnz,
                            "precision": "bf16 shadow factors, fp32 master and accumulation" if w.precision == "bf16" else "fp32",
                            "path": "sparse" if path == B.TSID_PATH_SPARSE else "dense_tc",
+                           "values": "one byte per rating" if args.values == "u8" else "fp32",
                            "step": "tsid_grad_step (eta=%g lambda=%g xi=%g clip=%d norm=%d/%d)" % (
                                w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q),
                            "l2": "L2 flushed between timed steps (resident set %.0f MB)" % (resident / 1e6) if flush

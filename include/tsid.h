@@ -95,7 +95,10 @@ typedef enum { TSID_NORM_NONE = 0, TSID_NORM_COUNT = 1 } tsid_norm_t;
 
 enum {
   TSID_VALIDATE = 1u,         /* also check Omega for duplicate (row, col) pairs            */
-  TSID_INPUT_ROW_SORTED = 2u  /* promise: COO is sorted by (row, col); checked, skips a sort */
+  TSID_INPUT_ROW_SORTED = 2u, /* promise: COO is sorted by (row, col); checked, skips a sort */
+  TSID_VALUES_U8 = 4u         /* promise: every value is an integer in [0, 255] (ratings); checked
+                                 (else TSID_ERR_UNSUPPORTED).  The gradient passes then stream one byte
+                                 per value instead of four; results are bitwise the same.            */
 };
 
 typedef struct {

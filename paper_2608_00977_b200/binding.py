@@ -25,7 +25,7 @@ TSID_F32, TSID_BF16_SHADOW = 0, 1
 TSID_PATH_AUTO, TSID_PATH_SPARSE, TSID_PATH_DENSE_TC = 0, 1, 2
 TSID_CLIP_NONE, TSID_CLIP_ASYM_STEP, TSID_CLIP_ASYM_GRAD, TSID_CLIP_ASYM_ENTRY = 0, 1, 2, 3
 TSID_NORM_NONE, TSID_NORM_COUNT = 0, 1
-TSID_VALIDATE, TSID_INPUT_ROW_SORTED = 1, 2
+TSID_VALIDATE, TSID_INPUT_ROW_SORTED, TSID_VALUES_U8 = 1, 2, 4
 
 # every symbol include/tsid.h declares
 EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "tsid_fit", "tsid_loss",

@@ -72,6 +72,10 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
   }
   t->rowside.ptr = t->row_ptr; t->rowside.idx = t->col_idx; t->rowside.val = t->val_csr;
   t->colside.ptr = t->col_ptr; t->colside.idx = t->row_idx; t->colside.val = t->val_csc;
+  if (c.flags & TSID_VALUES_U8) {
+    t->rowside.val8 = cv.take<uint8_t>(nz);
+    t->colside.val8 = cv.take<uint8_t>(nz);
+  }
   t->partial = cv.take<float>((2 * per + 2) * k);
   t->red_cap = (int32_t)(2 + 2 * 256 + t->rowside.cap_seg);
   t->red = cv.take<double>(t->red_cap);
@@ -163,6 +167,12 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
   e = build_segments(t, t->rowside, cfg->norm_p, ls);
   if (e == cudaSuccess) e = build_segments(t, t->colside, cfg->norm_q, ls);
   if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+  if (cfg->flags & TSID_VALUES_U8) {
+    int32_t bad = 0;
+    e = sparse_pack_values_u8(t, &bad);
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+    if (bad) { tsid_destroy(t); return fail(nullptr, TSID_ERR_UNSUPPORTED, "TSID_VALUES_U8 promised but a value is not an integer in [0, 255]"); }
+  }
   if (path == TSID_PATH_DENSE_TC) {
     int32_t bad = 0;
     e = dense_build(t, &bad);

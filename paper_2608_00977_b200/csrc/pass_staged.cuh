@@ -58,10 +58,11 @@ struct StagedMinBlocks {
   static constexpr int value = KP <= 64 ? 32 : (KP == 128 ? 18 : 1);
 };
 
-template <int KP, bool BF16, int NST, int ROWS, bool ENTRY>
+// V8: the values come as one byte each (integers 0..255) instead of fp32; the arithmetic is the same.
+template <int KP, bool BF16, int NST, int ROWS, bool ENTRY, bool V8>
 __global__ void __launch_bounds__(32, StagedMinBlocks<KP, BF16>::value)
 pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__restrict__ idx,
-                   const float *__restrict__ val, const void *__restrict__ stage_v,
+                   const void *__restrict__ val_v, const void *__restrict__ stage_v,
                    const void *__restrict__ gather_v, int k, float *__restrict__ G,
                    float *__restrict__ partial, float lam2, float xi) {
   using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
@@ -111,7 +112,8 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
   for (int i = 0; i < EPL; ++i) acc[i] = 0.f;
 
   const int32_t *ip = idx + sg.begin;
-  const float *vp = val + sg.begin;
+  const float *vp = static_cast<const float *>(val_v) + sg.begin;
+  const uint8_t *vp8 = static_cast<const uint8_t *>(val_v) + sg.begin;
   const int len = sg.len;
   const int nchunks = (len + ROWS - 1) / ROWS;
 
@@ -148,7 +150,10 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
   auto load_iv = [&](int c, int32_t &j, float &r) {
     j = 0;
     r = 0.f;
-    if (lane < ROWS && c * ROWS + lane < len) { j = __ldcs(ip + c * ROWS + lane); r = __ldcs(vp + c * ROWS + lane); }
+    if (lane < ROWS && c * ROWS + lane < len) {
+      j = __ldcs(ip + c * ROWS + lane);
+      r = V8 ? (float)__ldcs(vp8 + c * ROWS + lane) : __ldcs(vp + c * ROWS + lane);
+    }
   };
 
   // prologue: chunks 0 .. NST-2 in flight, indices of chunk NST-1 loaded
@@ -269,13 +274,21 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
   }
 }
 
-template <int KP, bool BF16, int NST, int ROWS, bool ENTRY>
+template <int KP, bool BF16, int NST, int ROWS, bool ENTRY, bool V8>
 cudaError_t launch_staged_t(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
   using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
   constexpr int smem = NST * ROWS * KP * (int)sizeof(T);
-  auto kern = pass_staged_kernel<KP, BF16, NST, ROWS, ENTRY>;
+  auto kern = pass_staged_kernel<KP, BF16, NST, ROWS, ENTRY, V8>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  kern<<<sd.nseg, 32, smem, t->stream>>>(sd.segs, sd.nseg, sd.idx, sd.val, stage, gather, t->cfg.k, G, t->partial,
+  const void *val = V8 ? static_cast<const void *>(sd.val8) : static_cast<const void *>(sd.val);
+  kern<<<sd.nseg, 32, smem, t->stream>>>(sd.segs, sd.nseg, sd.idx, val, stage, gather, t->cfg.k, G, t->partial,
                                          2.0f * t->cfg.lambda, t->cfg.xi);
   return cudaGetLastError();
+}
+
+// byte values when the side has them
+template <int KP, bool BF16, int NST, int ROWS, bool ENTRY>
+cudaError_t launch_staged_v(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G) {
+  if (sd.val8) return launch_staged_t<KP, BF16, NST, ROWS, ENTRY, true>(t, sd, stage, gather, G);
+  return launch_staged_t<KP, BF16, NST, ROWS, ENTRY, false>(t, sd, stage, gather, G);
 }

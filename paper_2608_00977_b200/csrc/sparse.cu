@@ -371,16 +371,16 @@ cudaError_t launch_staged_e(tsid_template *t, const Side &sd, const void *stage,
   if (sd.nseg <= 0) return cudaSuccess;
   const int k = t->cfg.k;
   if (t->cfg.precision == TSID_BF16_SHADOW) {
-    if (k <= 16) return launch_staged_t<16, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
-    if (k <= 32) return launch_staged_t<32, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
-    if (k <= 64) return launch_staged_t<64, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
-    if (k <= 128) return launch_staged_t<128, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
-    return launch_staged_t<256, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 16) return launch_staged_v<16, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 32) return launch_staged_v<32, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 64) return launch_staged_v<64, true, 2, 32, ENTRY>(t, sd, stage, gather, G);
+    if (k <= 128) return launch_staged_v<128, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
+    return launch_staged_v<256, true, 2, 16, ENTRY>(t, sd, stage, gather, G);
   }
-  if (k <= 16) return launch_staged_t<16, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
-  if (k <= 32) return launch_staged_t<32, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
-  if (k <= 64) return launch_staged_t<64, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
-  if (k <= 128) return launch_staged_t<128, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 16) return launch_staged_v<16, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 32) return launch_staged_v<32, false, 2, 32, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 64) return launch_staged_v<64, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
+  if (k <= 128) return launch_staged_v<128, false, 2, 16, ENTRY>(t, sd, stage, gather, G);
   return cudaErrorNotSupported;
 }
 
@@ -469,6 +469,32 @@ __global__ void scale_kernel(const int32_t *__restrict__ cnt, int32_t nrows, int
     const int32_t c = cnt[i];
     scale[i] = 2.0f / ((norm_count && c > 1) ? (float)c : 1.0f);
   }
+}
+
+// byte copies of the value streams; flags[FLAG_RANGE] if a value is not an integer in [0, 255]
+__global__ void pack_u8_kernel(const float *__restrict__ v, int64_t n, uint8_t *__restrict__ o, int32_t *flags) {
+  bool bad = false;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float x = v[i];
+    const int q = (int)x;
+    if (!(x >= 0.f && x <= 255.f) || (float)q != x) bad = true;
+    o[i] = (uint8_t)q;
+  }
+  if (bad) flags[FLAG_RANGE] = 1;
+}
+
+cudaError_t sparse_pack_values_u8(tsid_template *t, int32_t *h_bad) {
+  const int64_t nnz = t->cfg.nnz;
+  CK(cudaMemsetAsync(t->flags + FLAG_RANGE, 0, sizeof(int32_t), t->stream));
+  if (nnz > 0) {
+    pack_u8_kernel<<<ew_grid(nnz), 256, 0, t->stream>>>(t->rowside.val, nnz, const_cast<uint8_t *>(t->rowside.val8), t->flags);
+    pack_u8_kernel<<<ew_grid(nnz), 256, 0, t->stream>>>(t->colside.val, nnz, const_cast<uint8_t *>(t->colside.val8), t->flags);
+  }
+  CK(cudaGetLastError());
+  CK(cudaMemcpyAsync(h_bad, t->flags + FLAG_RANGE, sizeof(int32_t), cudaMemcpyDeviceToHost, t->stream));
+  CK(cudaStreamSynchronize(t->stream));
+  if (*h_bad) CK(cudaMemsetAsync(t->flags + FLAG_RANGE, 0, sizeof(int32_t), t->stream));
+  return cudaSuccess;
 }
 
 cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt) {

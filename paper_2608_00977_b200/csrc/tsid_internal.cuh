@@ -39,6 +39,7 @@ struct Side {
   const int64_t *ptr = nullptr;   // [nrows+1]
   const int32_t *idx = nullptr;   // [nnz] opposite-side index of each entry
   const float *val = nullptr;     // [nnz]
+  const uint8_t *val8 = nullptr;  // [nnz] the same values as bytes (TSID_VALUES_U8), else null
   Segment *segs = nullptr;
   SplitRow *splits = nullptr;
   float *scale = nullptr;  // [nrows] 2 / s_i
@@ -128,6 +129,7 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
 cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_Q, float *d_e);
 cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
 int sparse_launches_per_step(const tsid_template *t);
+cudaError_t sparse_pack_values_u8(tsid_template *t, int32_t *h_bad);
 cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt);
 cudaError_t sparse_scale_from_counts(tsid_template *t, Side &sd, int norm_mode, const int32_t *d_cnt);
 cudaError_t sparse_side_grad(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G);

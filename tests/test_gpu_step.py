@@ -217,3 +217,31 @@ def test_argument_errors():
     assert L.tsid_grad_step(None, None, None, None, None) == B.TSID_ERR_INVALID_ARG
     assert L.tsid_destroy(None) == B.TSID_OK
     assert b"epochs" in L.tsid_last_error(T.h)
+
+
+@pytest.mark.parametrize("precision,k", [("f32", 32), ("bf16", 64), ("bf16", 128)])
+def test_byte_value_streams_give_the_same_bits(precision, k):
+    """TSID_VALUES_U8: ratings streamed as one byte each.  Same arithmetic, so the same bits; a value that
+    is not an integer in [0, 255] is refused at create."""
+    w = small_workload("u8", 3000, 1700, k, 200_000, positions="zipf", precision=precision, seed=3 + k,
+                       values="ratings", eta=0.05, lam=0.03, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT,
+                       norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    assert float(tpl.vals.min()) >= 1 and float(tpl.vals.max()) <= 5
+    outs = []
+    for flags in (0, B.TSID_VALUES_U8):
+        T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE, flags=flags)
+        P, Q = tpl.P0.clone(), tpl.Q0.clone()
+        GP, GQ = torch.empty_like(P), torch.empty_like(Q)
+        T.tsid_grad_step(P, Q, GP, GQ)
+        T.tsid_grad_step(P, Q)
+        T.tsid_check()
+        outs.append((P, Q, GP, GQ))
+        T.tsid_destroy()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    bad = tpl.vals.clone()
+    bad[7] = 2.5
+    with pytest.raises(B.TsidError) as e:
+        B.Template(B.make_config(w.m, w.n, w.k, tpl.nnz, flags=B.TSID_VALUES_U8), tpl.rows, tpl.cols, bad)
+    assert e.value.status == B.TSID_ERR_UNSUPPORTED
