@@ -1,9 +1,9 @@
 // Staged variant of the gradient pass.  Included by sparse.cu inside its namespace, after Geo,
 // Raw and the pass_kernel it mirrors.
 //
-// Same arithmetic and the same summation order as pass_kernel<MODE_GRAD> (bitwise identical
-// results), but the gathered factor rows travel global -> shared memory with 16-byte asynchronous
-// copies (cp.async, L2 only), NST chunks of ROWS rows deep.  The bytes in flight then live in
+// Same arithmetic as pass_kernel<MODE_GRAD> (the dot products are summed as an even and an odd half
+// by packed fp32 FMAs, otherwise in the same order), but the gathered factor rows travel global ->
+// shared memory with 16-byte asynchronous copies (cp.async, L2 only), NST chunks of ROWS rows deep.  The bytes in flight then live in
 // shared memory instead of registers; the k = 128 passes are bound by exactly that (gathers served
 // by L2 / HBM at several hundred ns each, 256 B per entry).  A CTA is ONE warp: segments differ in
 // length, and a multi-warp CTA keeps the shared memory of its finished warps idle until its longest
@@ -200,19 +200,38 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
             float fa[EPL], fb[EPL];
 #pragma unroll
             for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
-            float da = 0.f, db = 0.f;
+            // two fp32 FMAs per instruction (sm_100 packed fp32): the dot products run as an even and an
+            // odd partial sum, the accumulation as pairs of coordinates
+            float2 da2 = make_float2(0.f, 0.f), db2 = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+            for (int i = 0; i < EPL; i += 2) {
+              const float2 x2 = make_float2(x[i], x[i + 1]);
+              da2 = __ffma2_rn(x2, make_float2(fa[i], fa[i + 1]), da2);
+              db2 = __ffma2_rn(x2, make_float2(fb[i], fb[i + 1]), db2);
+            }
+            float da = da2.x + da2.y, db = db2.x + db2.y;
 #pragma unroll
             for (int o = GROUP / 2; o > 0; o >>= 1) {
               da += __shfl_xor_sync(0xffffffffu, da, o);
               db += __shfl_xor_sync(0xffffffffu, db, o);
             }
             const float ea = ra - da, eb = rb - db;
+            if (ENTRY) {
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, true);
+              for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, true);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, true);
+              for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, true);
+            } else {
+              const float2 ea2 = make_float2(ea, ea), eb2 = make_float2(eb, eb);
+#pragma unroll
+              for (int i = 0; i < EPL; i += 2) {
+                float2 a2 = make_float2(acc[i], acc[i + 1]);
+                a2 = __ffma2_rn(ea2, make_float2(fa[i], fa[i + 1]), a2);
+                a2 = __ffma2_rn(eb2, make_float2(fb[i], fb[i + 1]), a2);
+                acc[i] = a2.x;
+                acc[i + 1] = a2.y;
+              }
+            }
           }
         } else {
           const int iters = (nv + EPW - 1) / EPW;
