@@ -86,3 +86,41 @@ def test_one_shard_equals_grad_step_bitwise():
         T.tsid_grad_step(Pb.view(-1), Qb.view(-1))
     assert torch.equal(Pa, Pb) and torch.equal(Qa, Qb)
     s.destroy(); T.tsid_destroy()
+
+
+def test_split_step_argument_errors_and_counts():
+    w = small_workload("shard-args", 300, 200, 8, 5_000, seed=9, norm_p=W.NORM_COUNT, norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV)
+    T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    L = B.lib()
+    P, Q = tpl.P0.clone(), tpl.Q0.clone()
+    GP, GQ = torch.empty_like(P), torch.empty_like(Q)
+    # null or misaligned gradient buffers are refused before any launch
+    assert L.tsid_grad(T.h, P.data_ptr(), Q.data_ptr(), None, GQ.data_ptr()) == B.TSID_ERR_INVALID_ARG
+    assert L.tsid_apply(T.h, P.data_ptr(), Q.data_ptr(), GP.data_ptr() + 4, GQ.data_ptr()) == B.TSID_ERR_INVALID_ARG
+    assert L.tsid_grad(None, P.data_ptr(), Q.data_ptr(), GP.data_ptr(), GQ.data_ptr()) == B.TSID_ERR_INVALID_ARG
+    assert L.tsid_get_counts(None, None, None) == B.TSID_ERR_INVALID_ARG
+    # counts are the row and column degrees of the template
+    cp, cq = T.tsid_get_counts()
+    rows, cols, _ = np_coo(tpl)
+    assert np.array_equal(cp.cpu().numpy(), np.bincount(rows, minlength=w.m))
+    assert np.array_equal(cq.cpu().numpy(), np.bincount(cols, minlength=w.n))
+    # grad + apply with the template's own counts is tsid_grad_step
+    T.tsid_set_norm_counts(cp, cq)
+    Pa, Qa = tpl.P0.clone(), tpl.Q0.clone()
+    T.tsid_grad(Pa, Qa, GP, GQ)
+    T.tsid_apply(Pa, Qa, GP, GQ)
+    T.tsid_grad_step(P, Q)
+    assert torch.equal(Pa, P) and torch.equal(Qa, Q)
+    # doubled column counts halve the normalised part of the column direction
+    T.tsid_set_norm_counts(None, cq * 2)
+    Pb, Qb = tpl.P0.clone(), tpl.Q0.clone()
+    T.tsid_grad(Pb, Qb, GP, GQ)
+    T.tsid_apply(Pb, Qb, GP, GQ)
+    ref = oracle.grad_step(w.m, w.n, w.k, rows, cols, np_coo(tpl)[2], tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy(),
+                           w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
+    s2 = np.where(2 * np.bincount(cols, minlength=w.n) > 1, 2 * np.bincount(cols, minlength=w.n), 1)[:, None]
+    Qexp = tpl.Q0.cpu().numpy().astype(np.float64) + w.eta * (2.0 * ref.GQ / s2 - 2.0 * w.lam * tpl.Q0.cpu().numpy())
+    assert relerr(Qb.cpu().numpy(), Qexp) <= F32_TOL
+    assert torch.equal(Pb, P)
+    T.tsid_destroy()
