@@ -64,7 +64,9 @@ def test_sampling_is_uniform_over_columns():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("m,n,nnz,alpha,seed", [(300, 200, 9000, 0.1, 1), (64, 5000, 40_000, 0.5, 2), (500, 37, 3000, 0.3, 3),
-                                               (100, 100, 0, 0.2, 4), (2000, 1500, 150_000, 1.0, 5), (50, 3, 120, 0.01, 6)])
+                                               (100, 100, 0, 0.2, 4), (2000, 1500, 150_000, 1.0, 5), (50, 3, 120, 0.01, 6),
+                                               (900, 300_000, 700_000, 0.37, 7),      # several tiles per block
+                                               (40, 2_500_000, 60_000, 0.5, 8)])      # bitmap too large for shared memory
 def test_gpu_sampling_is_bit_exact(m, n, nnz, alpha, seed):
     import torch
     from paper_2608_00977_b200 import binding as B
