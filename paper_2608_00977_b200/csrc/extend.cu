@@ -106,7 +106,7 @@ __device__ __forceinline__ float4 fetch4(const float *__restrict__ P, int row, i
 }
 
 template <int BN, bool B_NK, bool VEC, class Epi>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, BN == 64 ? 3 : 2)
 gemm_kernel(const float *__restrict__ A, const float *__restrict__ B, int M, int N, int K, int kper, Epi epi) {
   constexpr int TH = BN / 32;   // half of the thread's columns: 4 (BN = 128) or 2 (BN = 64)
   constexpr int NA = BM * BK / 4 / 256, NB = BN * BK / 4 / 256;   // float4 loads per thread and slice
