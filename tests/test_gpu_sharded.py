@@ -124,3 +124,39 @@ def test_split_step_argument_errors_and_counts():
     assert relerr(Qb.cpu().numpy(), Qexp) <= F32_TOL
     assert torch.equal(Pb, P)
     T.tsid_destroy()
+
+
+def test_sharded_dense_path():
+    """Row shards that run the tcgen05 variant: the split step and the sum of G_Q work the same way."""
+    m, n, k, world = 512, 384, 64, 2
+    w = W.Workload("shard-dense", m, n, k, int(0.3 * m * n), "bernoulli", density=0.30, seed=21, values="lowrank",
+                   noise_var=1e-4, precision="bf16", eta=0.2, lam=0.0, clip=W.CLIP_NONE, norm_p=W.NORM_COUNT,
+                   norm_q=W.NORM_COUNT, epochs=3)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    shards, Ps, Qs = [], [], []
+    for r in range(world):
+        r0, r1 = S.row_block(m, r, world)
+        rows, cols, vals = S.shard_coo(tpl.rows, tpl.cols, tpl.vals, r0, r1)
+        shards.append(S.RowShard(r1 - r0, n, k, rows, cols, vals, precision=B.TSID_BF16_SHADOW, path=B.TSID_PATH_DENSE_TC,
+                                 eta=w.eta, lam=w.lam, xi=w.xi, clip=w.clip, norm_p=w.norm_p, norm_q=w.norm_q))
+        assert shards[-1].T.tsid_get_info()[0] == B.TSID_PATH_DENSE_TC
+        Ps.append(tpl.P0[r0:r1].clone().contiguous())
+        Qs.append(tpl.Q0.clone())
+    cq = sum(s.col_counts.clone() for s in shards)
+    for s in shards:
+        s.set_global_col_counts(cq)
+    for s, P, Q in zip(shards, Ps, Qs):
+        s.grad(P, Q)
+    total = shards[0].GQ + shards[1].GQ
+    for s, P, Q in zip(shards, Ps, Qs):
+        s.GQ.copy_(total)
+        s.apply(P, Q)
+        s.T.tsid_check()
+    assert torch.equal(Qs[0], Qs[1])
+    rows, cols, vals = np_coo(tpl)
+    ref = oracle.grad_step(m, n, k, rows, cols, vals, tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy(), w.eta, w.lam, w.xi,
+                           w.clip, w.norm_p, w.norm_q, bf16_emulate=True)
+    assert relerr(total.view(n, k).cpu().numpy(), ref.GQ) <= 1e-2      # the dense path rounds E to bf16
+    assert relerr(torch.cat(Ps).cpu().numpy(), ref.P) <= 1e-3 and relerr(Qs[0].cpu().numpy(), ref.Q) <= 1e-3
+    for s in shards:
+        s.destroy()
