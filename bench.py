@@ -334,8 +334,25 @@ def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize(dev)
+    step = lambda: sh.step(P, Q)
+    if args.exchange == "peer":
+        # the exchange folded into the update kernel: G_Q parts and Q replicas mapped into every rank
+        if world > 1:
+            gq, gq_ptrs, gq_bar = S.symmetric_buffers(w.n * w.k, dev, dist)
+            qs, q_ptrs, q_bar = S.symmetric_buffers(w.n * w.k, dev, dist)
+            qs.copy_(Q.view(-1))
+            Q = qs.view(w.n, w.k)
+            sh.GQ = gq
+        else:
+            gq_ptrs, q_ptrs, gq_bar, q_bar = [sh.GQ.data_ptr()], [Q.data_ptr()], (lambda: None), (lambda: None)
+
+        def step():
+            sh.grad(P, Q)
+            gq_bar()                                   # all parts complete
+            sh.apply_sliced(P, q_ptrs, gq_ptrs, rank)
+            q_bar()                                    # all slices stored
     for _ in range(args.warmup):
-        sh.step(P, Q)
+        step()
     sh.T.tsid_check()
     sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
     sampler.start()
@@ -344,7 +361,7 @@ def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(stream)
     for _ in range(args.steps):
-        sh.step(P, Q)
+        step()
     b.record(stream)
     barrier()
     ms = max_over_ranks(a.elapsed_time(b), dist, dev)
@@ -358,7 +375,9 @@ def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
                           "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
                           "dtype": "bf16" if w.precision == "bf16" else "f32", "data": "synthetic",
                           "config": {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": tpl.nnz,
-                                     "parallelism": "rows/%d, all-reduce(sum) of G_Q (%d bytes) per step" % (world, w.n * w.k * 4),
+                                     "parallelism": ("rows/%d, exchange of G_Q (%d bytes) folded into the update kernel over peer memory"
+                                                     if args.exchange == "peer" else
+                                                     "rows/%d, all-reduce(sum) of G_Q (%d bytes) per step") % (world, w.n * w.k * 4),
                                      "l2": "inputs larger than L2, steps timed back to back"},
                           "clocks": clocks, "e2e": None, "gpu_launches": launches * args.steps, "roofline": None,
                           "cpu_baseline": None, "rmse_after": (sse / tpl.nnz) ** 0.5}))
@@ -383,6 +402,9 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
                     help="N > 1: independent replicas of the template (default), or ONE template sharded by rows "
                          "with one all-reduce of G_Q per step")
+    ap.add_argument("--exchange", default="nccl", choices=["nccl", "peer"],
+                    help="--shard rows: NCCL all-reduce of G_Q, or the exchange folded into the update kernel "
+                         "(tsid_apply_sliced over symmetric memory)")
     ap.add_argument("--values", default="f32", choices=["f32", "u8"],
                     help="u8: stream the ratings as one byte each (TSID_VALUES_U8; needs integer values, e.g. C2, C3, C5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

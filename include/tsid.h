@@ -156,6 +156,18 @@ tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *
 tsid_status_t tsid_grad(tsid_template_t *t, const float *d_P, const float *d_Q, float *d_GP, float *d_GQ);
 tsid_status_t tsid_apply(tsid_template_t *t, float *d_P, float *d_Q, const float *d_GP, const float *d_GQ);
 tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int32_t *d_cnt_q_or_null);
+/* tsid_apply with the exchange of G_Q folded into the update kernel (no counterpart in the paper).
+ * h_GQ_parts and h_Q_replicas are HOST arrays of `world` DEVICE pointers: part r is rank r's partial
+ * G_Q (n x k fp32, written by its tsid_grad), replica r is rank r's copy of Q; pointers of other ranks
+ * must be mapped into this process (peer access, symmetric or IPC memory) and are used with plain
+ * loads and stores only.  Updates P (this rank's rows) from d_GP, and the rows
+ * [n rank / world, n (rank + 1) / world) of Q: their parts are added in rank order, the update is
+ * applied once and the result is stored into EVERY replica.  The caller synchronises the ranks before
+ * the call (all parts complete) and after it (all slices stored) before anything reads Q or rewrites
+ * a part; the bf16 shadows are refreshed by the next tsid_grad.  world <= 16.  Asynchronous.
+ * Errors: TSID_ERR_INVALID_ARG. */
+tsid_status_t tsid_apply_sliced(tsid_template_t *t, float *d_P, const float *d_GP, float *const *h_Q_replicas,
+                                const float *const *h_GQ_parts, int32_t rank, int32_t world);
 tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or_null,
                                    const int32_t *d_cnt_q_or_null);
 

@@ -33,7 +33,7 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
-           "tsid_set_norm_counts"]
+           "tsid_set_norm_counts", "tsid_apply_sliced"]
 
 
 class TsidConfig(C.Structure):
@@ -79,6 +79,7 @@ def lib():
         L.tsid_apply.argtypes = [vp, vp, vp, vp, vp]
         L.tsid_get_counts.argtypes = [vp, vp, vp]
         L.tsid_set_norm_counts.argtypes = [vp, vp, vp]
+        L.tsid_apply_sliced.argtypes = [vp, vp, vp, C.POINTER(vp), C.POINTER(vp), C.c_int32, C.c_int32]
         L.tsid_loss.argtypes = [vp, vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.tsid_check.argtypes = [vp]
         L.tsid_destroy.argtypes = [vp]
@@ -185,6 +186,19 @@ class Template:
         _check_tensor(gradP, torch.float32, self.m * self.k, "gradP")
         _check_tensor(gradQ, torch.float32, self.n * self.k, "gradQ")
         st = lib().tsid_apply(self.h, P.data_ptr(), Q.data_ptr(), gradP.data_ptr(), gradQ.data_ptr())
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_apply_sliced(self, P, gradP, q_ptrs, gq_ptrs, rank):
+        """q_ptrs / gq_ptrs: device addresses (ints) of every rank's Q replica and partial G_Q."""
+        _check_tensor(P, torch.float32, self.m * self.k, "P")
+        _check_tensor(gradP, torch.float32, self.m * self.k, "gradP")
+        world = len(q_ptrs)
+        if len(gq_ptrs) != world:
+            raise ValueError("q_ptrs and gq_ptrs must have one entry per rank")
+        qa = (C.c_void_p * world)(*[int(x) for x in q_ptrs])
+        ga = (C.c_void_p * world)(*[int(x) for x in gq_ptrs])
+        st = lib().tsid_apply_sliced(self.h, P.data_ptr(), gradP.data_ptr(), qa, ga, int(rank), world)
         if st != TSID_OK:
             self._raise(st)
 

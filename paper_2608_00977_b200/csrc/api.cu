@@ -217,6 +217,20 @@ tsid_status_t tsid_apply(tsid_template_t *t, float *d_P, float *d_Q, const float
   return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
 }
 
+tsid_status_t tsid_apply_sliced(tsid_template_t *t, float *d_P, const float *d_GP, float *const *h_Q_replicas,
+                                const float *const *h_GQ_parts, int32_t rank, int32_t world) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (!d_P || !d_GP || !h_Q_replicas || !h_GQ_parts || !aligned16(d_P) || !aligned16(d_GP))
+    return fail(t, TSID_ERR_INVALID_ARG, "P, G_P and the pointer arrays must be non-null (P, G_P 16-byte aligned)");
+  if (world < 1 || world > kMaxRanks || rank < 0 || rank >= world)
+    return fail(t, TSID_ERR_INVALID_ARG, "need 1 <= world <= 16 and 0 <= rank < world");
+  for (int r = 0; r < world; ++r)
+    if (!h_Q_replicas[r] || !h_GQ_parts[r] || !aligned16(h_Q_replicas[r]) || !aligned16(h_GQ_parts[r]))
+      return fail(t, TSID_ERR_INVALID_ARG, "every Q replica and G_Q part must be a non-null, 16-byte aligned device pointer");
+  cudaError_t e = sparse_apply_sliced(t, d_P, d_GP, h_Q_replicas, h_GQ_parts, rank, world);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
+}
+
 tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int32_t *d_cnt_q_or_null) {
   if (!t) return TSID_ERR_INVALID_ARG;
   cudaError_t e = cudaSuccess;

@@ -256,6 +256,46 @@ update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int
   if (bad) flags[FLAG_NONFINITE] = 1;
 }
 
+// Exchange + update of one slice of Q for a row-sharded template, in one kernel.  The slice's rows of
+// every rank's partial G_Q are read with plain loads (this GPU's memory or a peer's mapped memory) and
+// added in rank order, the update is applied once, and the new values are stored with plain stores into
+// every rank's replica of Q: a reduce-scatter and an all-gather folded into the update, with no
+// intermediate buffer.  Since one rank computes a row and all receive the same bits, the replicas cannot
+// drift.  (No multicast and no waiting inside the kernel: the ranks synchronise before and after it.)
+constexpr int kMaxPeers = 16;
+struct PeerPtrs {
+  const float *gq[kMaxPeers];
+  float *q[kMaxPeers];
+};
+__global__ void __launch_bounds__(256)
+apply_slice_kernel(PeerPtrs pp, int world, int self, const float *__restrict__ scale, int64_t j0, int64_t j1, int k4,
+                   float eta, float lam2, float xi, int clip, float gmul, int32_t *flags) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  bool bad = false;
+  for (int64_t j = j0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < j1; j += stride) {
+    const float sc = __ldg(scale + j / k4) * gmul;
+    float4 gv = *(reinterpret_cast<const float4 *>(pp.gq[0]) + j);
+    for (int r = 1; r < world; ++r) {
+      const float4 a = *(reinterpret_cast<const float4 *>(pp.gq[r]) + j);
+      gv.x += a.x; gv.y += a.y; gv.z += a.z; gv.w += a.w;
+    }
+    const float4 x = reinterpret_cast<const float4 *>(pp.q[self])[j];
+    float xs[4] = {x.x, x.y, x.z, x.w};
+    const float gs[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float d = fmaf(gs[q], sc, -lam2 * xs[q]);
+      bad |= !isfinite(d);
+      d = clip_dir(d, xi, clip);
+      xs[q] = fmaf(eta, d, xs[q]);
+      bad |= !isfinite(xs[q]);
+    }
+    const float4 nx = make_float4(xs[0], xs[1], xs[2], xs[3]);
+    for (int r = 0; r < world; ++r) reinterpret_cast<float4 *>(pp.q[r])[j] = nx;
+  }
+  if (bad) flags[FLAG_NONFINITE] = 1;
+}
+
 __global__ void __launch_bounds__(256)
 convert_kernel(const float *__restrict__ A, __nv_bfloat16 *__restrict__ Ab, int64_t na4,
                const float *__restrict__ B, __nv_bfloat16 *__restrict__ Bb, int64_t nb4) {
@@ -503,6 +543,31 @@ cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt) {
 }
 cudaError_t sparse_scale_from_counts(tsid_template *t, Side &sd, int norm_mode, const int32_t *d_cnt) {
   scale_kernel<<<ew_grid(sd.nrows), 256, 0, t->stream>>>(d_cnt, sd.nrows, norm_mode == TSID_NORM_COUNT, sd.scale);
+  return cudaGetLastError();
+}
+
+// P side: the usual update from the local sums.  Q side: rows [n rank / world, n (rank + 1) / world) through
+// apply_slice_kernel.
+cudaError_t sparse_apply_sliced(tsid_template *t, float *d_P, const float *GP, float *const *h_Q, const float *const *h_GQ,
+                                int rank, int world) {
+  const tsid_config_t &c = t->cfg;
+  const bool entry = c.clip == TSID_CLIP_ASYM_ENTRY;
+  const float lam2 = entry ? 0.f : 2.0f * c.lambda, gmul = entry ? 0.5f : 1.0f;
+  const int clip = entry ? (int)TSID_CLIP_NONE : (int)c.clip;
+  UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4};
+  UpdSide none{nullptr, nullptr, nullptr, nullptr, 0};
+  prof_mark(t, EV_UPD0);
+  if (a.n4 > 0) update_kernel<<<ew_grid(a.n4), 256, 0, t->stream>>>(a, none, c.k / 4, c.eta, lam2, c.xi, clip, gmul, t->flags);
+  PeerPtrs pp;
+  for (int r = 0; r < kMaxPeers; ++r) { pp.gq[r] = nullptr; pp.q[r] = nullptr; }
+  for (int r = 0; r < world; ++r) { pp.gq[r] = h_GQ[r]; pp.q[r] = h_Q[r]; }
+  const int k4 = c.k / 4;
+  const int64_t r0 = (int64_t)c.n * rank / world, r1 = (int64_t)c.n * (rank + 1) / world;
+  if (r1 > r0)
+    apply_slice_kernel<<<ew_grid((r1 - r0) * k4), 256, 0, t->stream>>>(pp, world, rank, t->colside.scale, r0 * k4, r1 * k4,
+                                                                     k4, c.eta, lam2, c.xi, clip, gmul, t->flags);
+  prof_mark(t, EV_UPD1);
+  if (t->prof.on && t->prof.nsteps < kProfSteps) t->prof.nsteps++;
   return cudaGetLastError();
 }
 

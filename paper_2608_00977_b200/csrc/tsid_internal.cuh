@@ -130,6 +130,9 @@ cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_
 cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
 int sparse_launches_per_step(const tsid_template *t);
 cudaError_t sparse_pack_values_u8(tsid_template *t, int32_t *h_bad);
+cudaError_t sparse_apply_sliced(tsid_template *t, float *d_P, const float *GP, float *const *h_Q, const float *const *h_GQ,
+                                int rank, int world);
+constexpr int kMaxRanks = 16;
 cudaError_t sparse_counts(tsid_template *t, const Side &sd, int32_t *d_cnt);
 cudaError_t sparse_scale_from_counts(tsid_template *t, Side &sd, int norm_mode, const int32_t *d_cnt);
 cudaError_t sparse_side_grad(tsid_template *t, const Side &sd, const void *stage, const void *gather, float *G);

@@ -35,6 +35,17 @@ def all_reduce_sum(t: torch.Tensor, dist=None, group=None) -> torch.Tensor:
     return t
 
 
+def symmetric_buffers(numel: int, device, dist, group=None):
+    """A float32 buffer of `numel` elements on every rank of `group`, each mapped into all the others
+    (torch's symmetric memory).  Returns (tensor, [device address on rank 0, rank 1, ...], barrier()).
+    Needs one process per GPU with peer access; this build had one GPU per call, so this helper has not run
+    on more than one GPU: the single-GPU tests pass the addresses of ordinary tensors instead."""
+    import torch.distributed._symmetric_memory as symm_mem
+    t = symm_mem.empty(numel, dtype=torch.float32, device=device)
+    hdl = symm_mem.rendezvous(t, group if group is not None else dist.group.WORLD)
+    return t, [int(p) for p in hdl.buffer_ptrs], hdl.barrier
+
+
 class RowShard:
     """One rank's part of a row-sharded template: a library template over its rows, the gradient buffers
     and the exchange.  `rows`, `cols`, `vals` are this rank's entries with LOCAL row numbers."""
@@ -68,6 +79,13 @@ class RowShard:
         self.grad(P_local, Q)
         all_reduce_sum(self.GQ, self.dist, self.group)
         self.apply(P_local, Q)
+
+    def apply_sliced(self, P_local, q_ptrs, gq_ptrs, rank):
+        """The exchange folded into the update kernel: this rank adds the partial G_Q of all ranks for its
+        slice of Q's rows (plain loads through the given device addresses), updates the slice once and
+        stores it into every replica; P is updated from the local sums.  The caller synchronises the ranks
+        before (all tsid_grad done) and after (all slices stored)."""
+        self.T.tsid_apply_sliced(P_local, self.GP, q_ptrs, gq_ptrs, rank)
 
     def sse(self, P_local, Q) -> float:
         """Sum of squared residuals over ALL ranks' entries."""

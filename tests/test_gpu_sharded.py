@@ -160,3 +160,56 @@ def test_sharded_dense_path():
     assert relerr(torch.cat(Ps).cpu().numpy(), ref.P) <= 1e-3 and relerr(Qs[0].cpu().numpy(), ref.Q) <= 1e-3
     for s in shards:
         s.destroy()
+
+
+@pytest.mark.parametrize("case", ["clip-count", "paper-literal", "bf16"])
+@pytest.mark.parametrize("world", [2, 3])
+def test_update_with_the_exchange_folded_in(case, world):
+    """tsid_apply_sliced: every emulated rank reduces and updates its slice of Q and stores it into all
+    replicas.  With all replicas and parts on one GPU the 'peer' addresses are ordinary device addresses."""
+    kw = CASES[case]
+    m, n, k, nnz, steps = 1203, 650, 32, 90_000, 3
+    w = small_workload("fused-" + case, m, n, k, nnz, positions="zipf", seed=31 + world, **kw)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    shards, Ps, Qs = [], [], []
+    for r in range(world):
+        r0, r1 = S.row_block(m, r, world)
+        rows, cols, vals = S.shard_coo(tpl.rows, tpl.cols, tpl.vals, r0, r1)
+        shards.append(S.RowShard(r1 - r0, n, k, rows, cols, vals, precision=prec, eta=w.eta, lam=w.lam, xi=w.xi,
+                                 clip=w.clip, norm_p=w.norm_p, norm_q=w.norm_q))
+        Ps.append(tpl.P0[r0:r1].clone().contiguous())
+        Qs.append(tpl.Q0.clone())
+    cq = sum(s.col_counts.clone() for s in shards)
+    for s in shards:
+        s.set_global_col_counts(cq)
+    q_ptrs = [Q.data_ptr() for Q in Qs]
+    gq_ptrs = [s.GQ.data_ptr() for s in shards]
+    for _ in range(steps):
+        for s, P, Q in zip(shards, Ps, Qs):
+            s.grad(P, Q)
+        torch.cuda.synchronize()                       # "all parts complete"
+        for r, (s, P) in enumerate(zip(shards, Ps)):
+            s.apply_sliced(P, q_ptrs, gq_ptrs, r)
+        torch.cuda.synchronize()                       # "all slices stored"
+        for s in shards:
+            s.T.tsid_check()
+    for Q in Qs[1:]:
+        assert torch.equal(Q, Qs[0])
+    rows, cols, vals = np_coo(tpl)
+    bf = w.precision == "bf16"
+    Pr, Qr, _ = oracle.fit(m, n, k, rows, cols, vals, tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy(), steps, w.eta, w.lam,
+                           w.xi, w.clip, w.norm_p, w.norm_q, bf16_emulate=bf, history=False)
+    tol = 2e-3 if bf else F32_TOL
+    assert relerr(torch.cat(Ps).cpu().numpy(), Pr) <= tol and relerr(Qs[0].cpu().numpy(), Qr) <= tol
+    # argument checks
+    L = B.lib()
+    T = shards[0].T
+    import ctypes as C
+    qa = (C.c_void_p * world)(*q_ptrs); ga = (C.c_void_p * world)(*gq_ptrs)
+    assert L.tsid_apply_sliced(T.h, Ps[0].data_ptr(), shards[0].GP.data_ptr(), qa, ga, world, world) == B.TSID_ERR_INVALID_ARG
+    assert L.tsid_apply_sliced(T.h, Ps[0].data_ptr(), shards[0].GP.data_ptr(), qa, ga, 0, 17) == B.TSID_ERR_INVALID_ARG
+    ga[1] = None
+    assert L.tsid_apply_sliced(T.h, Ps[0].data_ptr(), shards[0].GP.data_ptr(), qa, ga, 0, world) == B.TSID_ERR_INVALID_ARG
+    for s in shards:
+        s.destroy()
