@@ -297,7 +297,7 @@ def measure_extend(args, w, tpl, B, dev):
         Ch.zero_()
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
-        B.tsid_extend(P, Q, col_ptr, rows, vals, Ch, chunk, iters, 0.02, 0.05, cold_start=True)
+        B.tsid_extend(P, Q, col_ptr, rows, vals, Ch, chunk, iters, 0.02, 0.05, cold_start=True, tensor_cores=args.extend_tc)
         torch.cuda.synchronize(dev)
         if it >= args.warmup:
             times.append(time.perf_counter() - t0)
@@ -311,7 +311,9 @@ def measure_extend(args, w, tpl, B, dev):
     print(json.dumps({"metric": "Stage II observed-entry Adam updates/sec", "value": nnz * iters / t, "unit": "updates/s",
                       "s_per_call": t, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
                       "config": {"workload": w.name, "m": w.m, "n_cols": w.n, "d": d, "k": w.k, "nnz": nnz,
-                                 "iters": iters, "chunk_cols": chunk, "dtype": "f32"},
+                                 "iters": iters, "chunk_cols": chunk,
+                                 "dtype": "bf16 operands / fp32 accumulation for the gradient product, fp32 elsewhere"
+                                          if args.extend_tc else "f32"},
                       "h2d_bytes_per_call": nnz * 8 + (w.n + 1) * 8, "d2h_bytes_per_call": w.n * d * 4,
                       "roofline": {"bound": "hbm", "achieved": alg_dev / t / 1e9, "peak": peak, "unit": "GB/s",
                                    "frac": alg_dev / t / 1e9 / peak, "alg_bytes": alg_dev,
@@ -402,6 +404,8 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
                     help="N > 1: independent replicas of the template (default), or ONE template sharded by rows "
                          "with one all-reduce of G_Q per step")
+    ap.add_argument("--extend-tc", action="store_true",
+                    help="--measure extend: the gradient product on the tensor cores (TSID_EXTEND_TC, mixed precision)")
     ap.add_argument("--exchange", default="nccl", choices=["nccl", "peer"],
                     help="--shard rows: NCCL all-reduce of G_Q, or the exchange folded into the update kernel "
                          "(tsid_apply_sliced over symmetric memory)")

@@ -386,11 +386,11 @@ def tsid_sample_template(m, n, rows, cols, vals, alpha, seed, stream=None):
     return colmap, ro[:k], co[:k], vo[:k], d.value
 
 
-TSID_EXTEND_COLD_START = 1
+TSID_EXTEND_COLD_START, TSID_EXTEND_TC = 1, 2
 
 
 def tsid_extend(P, Q, col_ptr, row_idx, vals, C0, chunk_cols, iters, eta, lam, beta1=0.9, beta2=0.999, eps=1e-8,
-                want_sse=False, stream=None, cold_start=False):
+                want_sse=False, stream=None, cold_start=False, tensor_cores=False):
     """Stage II extension.  P (m x k), Q (d x k): CUDA fp32 tensors.  col_ptr (int64), row_idx (int32),
     vals (fp32), C0 (fp32 [n_cols, d]): CPU tensors (pinned for asynchronous copies); C0 is overwritten with
     the fitted coefficients.  Returns the SSE if requested."""
@@ -407,7 +407,8 @@ def tsid_extend(P, Q, col_ptr, row_idx, vals, C0, chunk_cols, iters, eta, lam, b
     dev = P.device
     stream = stream if stream is not None else torch.cuda.current_stream(dev)
     cfg = TsidExtendConfig(m, d, k, n_cols, chunk_cols, iters, eta, lam, beta1, beta2, eps,
-                           TSID_EXTEND_COLD_START if cold_start else 0, stream.cuda_stream, None, 0)
+                           (TSID_EXTEND_COLD_START if cold_start else 0) | (TSID_EXTEND_TC if tensor_cores else 0),
+                           stream.cuda_stream, None, 0)
     need = C.c_size_t(0)
     st = lib().tsid_extend_workspace_bytes(C.byref(cfg), col_ptr.data_ptr(), C.byref(need))
     if st != TSID_OK:

@@ -33,10 +33,6 @@ namespace {
 constexpr int BM = 128, BK = 16;   // BN (128 or 64) is a template parameter
 constexpr int kSplitW = 8;         // K-splits of the tall-skinny first GEMM (K = d is long, M x N is small)
 
-struct AdamArgs {
-  float lr, lam2, b1, b2, eps, c1, c2;   // c1 = 1/(1-b1^t), c2 = 1/(1-b2^t)
-};
-
 struct SplitEpi {       // partial[z][m][n] = acc   (z = K-split index; summed in order by sum_splits_kernel)
   float *part;
   size_t plane;
@@ -202,6 +198,13 @@ gemm_kernel(const float *__restrict__ A, const float *__restrict__ B, int M, int
   }
 }
 
+__global__ void store_flag_kernel(const int32_t *flag, uint32_t *out) {
+  if (threadIdx.x == 0) {
+    *out = (uint32_t)*flag;
+    __threadfence_system();
+  }
+}
+
 // W = sum of the K-split partial planes, in split order
 __global__ void sum_splits_kernel(const float *__restrict__ part, size_t plane, int nsplit, float *__restrict__ W) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (size_t)gridDim.x * blockDim.x) {
@@ -237,6 +240,7 @@ struct ExtCarve {
   Segment *segs;
   SplitRow *splits;
   float *scale, *partial, *Mo, *Vo, *W, *U, *Wpart;
+  __nv_bfloat16 *Qb;    // [d * k] bf16 copy of Q (tensor-core form) or null
   double *red, *sse;
   int32_t *flags;
   LayoutScratch ls;
@@ -268,6 +272,7 @@ ExtCarve carve(void *base, const tsid_extend_config_t &c, int64_t cap) {
   e.W = cv.take<float>(cc * k);
   e.U = cv.take<float>(cc * k);
   e.Wpart = cv.take<float>((size_t)kSplitW * cc * k);
+  e.Qb = (c.flags & TSID_EXTEND_TC) ? cv.take<__nv_bfloat16>(d * k) : nullptr;
   e.red = cv.take<double>(2 + 2 * 256 + (size_t)e.cap_seg);
   e.sse = cv.take<double>(1);
   e.flags = cv.take<int32_t>(FLAG_COUNT);
@@ -285,6 +290,7 @@ tsid_status_t check(const tsid_extend_config_t *c, const int64_t *h_col_ptr, int
   if (!c || !h_col_ptr) return TSID_ERR_INVALID_ARG;
   if (c->m < 1 || c->d < 1 || c->n_cols < 1 || c->chunk_cols < 1 || c->iters < 0) return TSID_ERR_INVALID_ARG;
   if (c->k < 4 || c->k > 128 || (c->k & 3)) return TSID_ERR_UNSUPPORTED;
+  if ((c->flags & TSID_EXTEND_TC) && !extend_tc_qualifies(c->d, c->k)) return TSID_ERR_UNSUPPORTED;
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
     return TSID_ERR_INVALID_ARG;
   int64_t cap = 0;
@@ -326,6 +332,19 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
   ExtCarve e = carve(cfg->workspace, *cfg, cap);
   if (cfg->workspace_bytes < e.bytes) return TSID_ERR_OOM;
   const int32_t d = cfg->d, k = cfg->k, cc = cfg->chunk_cols;
+  // 64 bytes of pinned, device-mapped host memory for the words that come back every chunk (see LayoutScratch)
+  uint32_t *hmap = nullptr, *hmap_dev = nullptr;
+  if (cudaHostAlloc(reinterpret_cast<void **>(&hmap), 64, cudaHostAllocMapped) != cudaSuccess ||
+      cudaHostGetDevicePointer(reinterpret_cast<void **>(&hmap_dev), hmap, 0) != cudaSuccess) {
+    if (hmap) cudaFreeHost(hmap);
+    (void)cudaGetLastError();
+    return TSID_ERR_CUDA;
+  }
+  memset(hmap, 0, 64);
+  e.ls.hmap = hmap;
+  e.ls.hmap_dev = hmap_dev;
+  const bool use_tc = (cfg->flags & TSID_EXTEND_TC) != 0;   // check() made sure the shape qualifies
+  alignas(64) unsigned char tm_q[128];                     // tensor map of the bf16 copy of Q
 
   // a template object that only carries what the pass launchers read
   tsid_template ctx;
@@ -376,11 +395,10 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
     side.nrows = nc; side.ptr = e.ptr; side.idx = sl.rows; side.val = sl.vals;
     side.segs = e.segs; side.splits = e.splits; side.scale = e.scale;
     side.cap_seg = e.cap_seg; side.cap_split = e.cap_split; side.cap_slot = e.cap_slot;
+    // the range flag rides along with the segment totals (same host-mapped words, same synchronisation)
+    store_flag_kernel<<<1, 32, 0, s_cmp>>>(e.flags + FLAG_RANGE, e.ls.hmap_dev + 8);
     CK(build_segments(&ctx, side, TSID_NORM_NONE, e.ls));   // synchronises the compute stream
-    int32_t hf[FLAG_COUNT];
-    CK(cudaMemcpyAsync(hf, e.flags, sizeof(hf), cudaMemcpyDeviceToHost, s_cmp));
-    CK(cudaStreamSynchronize(s_cmp));
-    if (hf[FLAG_RANGE]) return cudaErrorInvalidValue;
+    if (e.ls.hmap[8]) return cudaErrorInvalidValue;
     const size_t cd = (size_t)nc * d;
     CK(cudaMemsetAsync(e.Mo, 0, sizeof(float) * cd, s_cmp));
     CK(cudaMemsetAsync(e.Vo, 0, sizeof(float) * cd, s_cmp));
@@ -405,7 +423,8 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
       p1 *= cfg->beta1; p2 *= cfg->beta2;
       AdamArgs aa{cfg->eta, 2.f * cfg->lambda, cfg->beta1, cfg->beta2, cfg->eps, (float)(1.0 / (1.0 - p1)),
                   (float)(1.0 / (1.0 - p2))};
-      if (vec) gemm_kernel<128, true, true, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
+      if (use_tc) CK(extend_tc_adam(s_cmp, e.U, tm_q, nc, d, k, sl.CT, e.Mo, e.Vo, aa, e.flags));
+      else if (vec) gemm_kernel<128, true, true, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
       else gemm_kernel<128, true, false, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
     }
     if (h_sse_or_null) {
@@ -416,10 +435,17 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
     CK(cudaEventRecord(cmp_done, s_cmp));
     // coefficients of this chunk go home on the third stream
     CK(cudaStreamWaitEvent(s_out, cmp_done, 0));
-    CK(cudaMemcpyAsync(h_C + (size_t)j0 * d, sl.CT, sizeof(float) * cd, cudaMemcpyDeviceToHost, s_out));
+    // in pieces: the few-byte reads of the next chunk's layout (segment totals, flags) go through the same
+    // copy engine and would otherwise queue behind this whole transfer, holding the compute stream up
+    const size_t piece = (size_t)2 << 20;   // floats: 8 MB per copy
+    for (size_t off = 0; off < cd; off += piece) {
+      const size_t cnt_f = cd - off < piece ? cd - off : piece;
+      CK(cudaMemcpyAsync(h_C + (size_t)j0 * d + off, sl.CT + off, sizeof(float) * cnt_f, cudaMemcpyDeviceToHost, s_out));
+    }
     return cudaEventRecord(sl.out_done, s_out);
   };
 
+  if (err == cudaSuccess && use_tc) err = extend_tc_prepare(s_cmp, d_Q, d, k, e.Qb, tm_q);
   if (err == cudaSuccess) err = cudaMemsetAsync(e.flags, 0, sizeof(int32_t) * FLAG_COUNT, s_cmp);
   if (err == cudaSuccess) err = cudaMemsetAsync(e.sse, 0, sizeof(double), s_cmp);
   if (err == cudaSuccess) err = cudaStreamSynchronize(s_cmp);
@@ -433,7 +459,10 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
   double sse = 0.0;
   if (err == cudaSuccess && h_sse_or_null)
     err = cudaMemcpyAsync(&sse, e.sse, sizeof(double), cudaMemcpyDeviceToHost, s_cmp);
+  int32_t hflags[FLAG_COUNT] = {0};
+  if (err == cudaSuccess) err = cudaMemcpyAsync(hflags, e.flags, sizeof(hflags), cudaMemcpyDeviceToHost, s_cmp);
   cudaError_t e2 = cudaStreamSynchronize(s_cmp);
+  if (hflags[FLAG_TIMEOUT] && err == cudaSuccess) err = cudaErrorLaunchTimeout;   // a bounded device-side wait expired
   cudaError_t e3 = s_out ? cudaStreamSynchronize(s_out) : cudaSuccess;
   cudaError_t e4 = s_in ? cudaStreamSynchronize(s_in) : cudaSuccess;
   if (h_sse_or_null) *h_sse_or_null = sse;
@@ -442,6 +471,7 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
     if (e.slot[s].out_done) cudaEventDestroy(e.slot[s].out_done);
   }
   if (cmp_done) cudaEventDestroy(cmp_done);
+  cudaFreeHost(hmap);
   if (s_in) cudaStreamDestroy(s_in);
   if (s_out) cudaStreamDestroy(s_out);
   if (bad_index) { (void)cudaGetLastError(); return TSID_ERR_INDEX_RANGE; }

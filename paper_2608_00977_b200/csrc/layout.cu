@@ -426,6 +426,14 @@ __global__ void seg_fill_kernel(const int64_t *__restrict__ ptr, int32_t nrows,
   }
 }
 
+// three words to a host-mapped buffer (visible to the host once the stream has been synchronised)
+__global__ void store3_kernel(const uint32_t *a, const uint32_t *b, const uint32_t *c, uint32_t *out) {
+  if (threadIdx.x == 0) {
+    out[0] = *a; out[1] = *b; out[2] = *c;
+    __threadfence_system();
+  }
+}
+
 inline int grid_for(int64_t n, int threads) {
   int64_t g = (n + threads - 1) / threads;
   if (g < 1) g = 1;
@@ -505,10 +513,17 @@ cudaError_t build_segments(tsid_template *t, Side &side, int norm_mode, LayoutSc
   CK(exclusive_scan_u32(s.scanB, s.scanB, nr, s, st));
   CK(exclusive_scan_u32(s.scanC, s.scanC, nr, s, st));
   uint32_t tot[3];
-  CK(cudaMemcpyAsync(&tot[0], s.scanA + nr, 4, cudaMemcpyDeviceToHost, st));
-  CK(cudaMemcpyAsync(&tot[1], s.scanB + nr, 4, cudaMemcpyDeviceToHost, st));
-  CK(cudaMemcpyAsync(&tot[2], s.scanC + nr, 4, cudaMemcpyDeviceToHost, st));
-  CK(cudaStreamSynchronize(st));
+  if (s.hmap_dev) {
+    store3_kernel<<<1, 32, 0, st>>>(s.scanA + nr, s.scanB + nr, s.scanC + nr, s.hmap_dev);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(st));
+    tot[0] = s.hmap[0]; tot[1] = s.hmap[1]; tot[2] = s.hmap[2];
+  } else {
+    CK(cudaMemcpyAsync(&tot[0], s.scanA + nr, 4, cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(&tot[1], s.scanB + nr, 4, cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(&tot[2], s.scanC + nr, 4, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+  }
   side.nseg = (int32_t)tot[0];
   side.nslot = (int32_t)tot[1];
   side.nsplit = (int32_t)tot[2];

@@ -108,6 +108,11 @@ struct LayoutScratch {
   uint32_t *hist;               // [256 * kSortBlocks]
   uint32_t *scanA, *scanB, *scanC;  // [max(m,n)+1] each
   uint32_t *blocksums;          // [kScanBlocksMax]
+  // Optional 64-byte pinned host buffer mapped into the device (host address, device alias).  When set,
+  // the few words the host needs back (segment totals, flags) are stored there by a kernel instead of
+  // going through the copy engine, where they would queue behind any large device-to-host transfer
+  // already submitted on another stream.
+  uint32_t *hmap = nullptr, *hmap_dev = nullptr;
 };
 constexpr int kSortBlocksMax = 148 * 6;
 constexpr int kScanBlocksMax = 1 << 20;
@@ -121,6 +126,15 @@ cudaError_t sort_pairs_u32(const uint32_t *kin, const uint32_t *vin, int64_t n, 
                            cudaStream_t st, uint32_t **kres, uint32_t **vres);
 // out[0..n) = exclusive scan of in[0..n), out[n] = total; in[n] must be 0; in may alias out
 cudaError_t scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch &s, cudaStream_t st);
+
+// Stage II (extend.cu, extend_tc.cu)
+struct AdamArgs {
+  float lr, lam2, b1, b2, eps, c1, c2;   // c1 = 1/(1-b1^t), c2 = 1/(1-b2^t)
+};
+bool extend_tc_qualifies(int32_t d, int32_t k);
+cudaError_t extend_tc_prepare(cudaStream_t st, const float *d_Q, int32_t d, int32_t k, __nv_bfloat16 *qb, void *tm);
+cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const void *tm, int32_t nc, int32_t d, int32_t k, float *Cm,
+                           float *Mo, float *Vo, const AdamArgs &aa, int32_t *flags);
 
 // sparse passes (sparse.cu)
 cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);

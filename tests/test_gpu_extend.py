@@ -82,3 +82,36 @@ def test_extend_errors():
     import ctypes as C
     need = C.c_size_t(0)
     assert B.lib().tsid_extend_workspace_bytes(C.byref(cfg), torch.tensor(cp).data_ptr(), C.byref(need)) == B.TSID_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("m,d,k,ncols,per_col,chunk", [(800, 200, 64, 257, 80, 100), (600, 260, 128, 300, 70, 150),
+                                                       (900, 1028, 64, 700, 90, 333)])
+def test_extend_tensor_core_form(m, d, k, ncols, per_col, chunk):
+    """TSID_EXTEND_TC: the gradient product on the tensor cores with bf16 operands (the paper's mixed
+    precision).  Adam turns a gradient coordinate into a step of about +-eta whatever its size, so where the
+    gradient is smaller than bf16's rounding the two precisions may step in opposite directions: the
+    coefficients are compared in the mean, the fit exactly, and the product itself through a run whose eps
+    is so large that the step is proportional to the gradient."""
+    P, Q, cp, ri, v = _problem(m, d, k, ncols, per_col, seed=m + d + k)
+    args = (torch.tensor(P, device=DEV), torch.tensor(Q, device=DEV), torch.tensor(cp).pin_memory(),
+            torch.tensor(ri).pin_memory(), torch.tensor(v).pin_memory())
+    Ch = torch.zeros(ncols, d).pin_memory()
+    # (1) eps = 1e4 >> |g|: one step from C = 0 gives C = -eta g / eps up to 1e-4 relative: the product itself
+    B.tsid_extend(*args, Ch, chunk, 1, 1.0, 0.05, eps=1e4, tensor_cores=True)
+    Cr, _ = oracle.extend(m, d, k, cp, ri, v, P, Q, 1.0, 0.05, 1, eps=1e4)
+    assert relerr(Ch.numpy(), Cr) <= 1e-2, relerr(Ch.numpy(), Cr)       # bf16 operands, fp32 accumulation
+    # (2) the fit
+    eta, lam, iters = 0.02, 0.05, 12
+    Ch.zero_()
+    sse_tc = B.tsid_extend(*args, Ch, chunk, iters, eta, lam, want_sse=True, tensor_cores=True)
+    C_tc = Ch.numpy().copy()
+    Cr, sse_r = oracle.extend(m, d, k, cp, ri, v, P, Q, eta, lam, iters)
+    rms = float(np.sqrt(np.mean((C_tc - Cr) ** 2)) / np.sqrt(np.mean(Cr ** 2)))
+    assert rms <= 0.1, rms
+    assert abs(sse_tc - sse_r) / sse_r <= 1e-3
+    assert not C_tc[min(3, ncols - 1)].any()
+    # a shape the tensor-core form does not take is refused, not silently run another way
+    with pytest.raises(B.TsidError) as e:
+        B.tsid_extend(torch.tensor(P[:, :32].copy(), device=DEV), torch.tensor(Q[:, :32].copy(), device=DEV), *args[2:], Ch,
+                      chunk, 1, eta, lam, tensor_cores=True)
+    assert e.value.status == B.TSID_ERR_UNSUPPORTED
