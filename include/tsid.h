@@ -264,10 +264,11 @@ tsid_status_t tsid_sample_template(int32_t m, int32_t n, int64_t nnz, double alp
  * UNSUPPORTED (k), OOM (workspace), INDEX_RANGE (a row index outside [0, m)), CUDA. */
 enum {
   TSID_EXTEND_COLD_START = 1u,   /* start from C = 0, h_C is only written */
-  TSID_EXTEND_TC = 2u            /* mixed precision as in the paper's Stage II (Sec. 5.2): the gradient product
-                                    U Q^T runs on the tensor cores with U and Q rounded to bf16 and fp32
-                                    accumulation; C and the Adam moments stay fp32.  Needs k in {64, 128},
-                                    d a multiple of 4 and >= 128 (else TSID_ERR_UNSUPPORTED). */
+  TSID_EXTEND_TC = 2u            /* mixed precision as in the paper's Stage II (Sec. 5.2): both products of a
+                                    step (W = C Q and U Q^T) run on the tensor cores with bf16 operands and
+                                    fp32 accumulation; C and the Adam moments stay fp32 (a bf16 copy of C is
+                                    kept beside it).  Needs k in {64, 128}, d a multiple of 8 and >= 128
+                                    (else TSID_ERR_UNSUPPORTED). */
 };
 typedef struct {
   int32_t m, d, k;     /* rows; template columns (rows of Q); rank                      */

@@ -231,6 +231,8 @@ struct Slot {           // buffers of one chunk in flight
   int32_t *rows;        // [cap]
   float *vals;          // [cap]
   float *CT;            // [cc * d]
+  __nv_bfloat16 *Cb;    // [cc * d] bf16 copy of CT (tensor-core form) or null
+  alignas(64) unsigned char mapC[128];   // its tensor map (host copy)
   cudaEvent_t in_done, out_done;
 };
 
@@ -257,6 +259,7 @@ ExtCarve carve(void *base, const tsid_extend_config_t &c, int64_t cap) {
     e.slot[s].rows = cv.take<int32_t>(cp);
     e.slot[s].vals = cv.take<float>(cp);
     e.slot[s].CT = cv.take<float>(cc * d);
+    e.slot[s].Cb = (c.flags & TSID_EXTEND_TC) ? cv.take<__nv_bfloat16>(cc * d) : nullptr;
   }
   e.ptr = cv.take<int64_t>(cc + 1);
   const size_t per = cp / kSegLen;
@@ -344,7 +347,7 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
   e.ls.hmap = hmap;
   e.ls.hmap_dev = hmap_dev;
   const bool use_tc = (cfg->flags & TSID_EXTEND_TC) != 0;   // check() made sure the shape qualifies
-  alignas(64) unsigned char tm_q[128];                     // tensor map of the bf16 copy of Q
+  ExtendTcMaps tc_maps;                                     // tensor maps of the bf16 copy of Q
 
   // a template object that only carries what the pass launchers read
   tsid_template ctx;
@@ -377,10 +380,13 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
       CK(cudaMemcpyAsync(sl.rows, h_row_idx + p0, sizeof(int32_t) * (size_t)cnt, cudaMemcpyHostToDevice, s_in));
       CK(cudaMemcpyAsync(sl.vals, h_vals + p0, sizeof(float) * (size_t)cnt, cudaMemcpyHostToDevice, s_in));
     }
-    if (cfg->flags & TSID_EXTEND_COLD_START)
+    if (cfg->flags & TSID_EXTEND_COLD_START) {
       CK(cudaMemsetAsync(sl.CT, 0, sizeof(float) * (size_t)(j1 - j0) * d, s_in));
-    else
+      if (use_tc) CK(cudaMemsetAsync(sl.Cb, 0, sizeof(__nv_bfloat16) * (size_t)(j1 - j0) * d, s_in));
+    } else {
       CK(cudaMemcpyAsync(sl.CT, h_C + (size_t)j0 * d, sizeof(float) * (size_t)(j1 - j0) * d, cudaMemcpyHostToDevice, s_in));
+      if (use_tc) CK(extend_tc_to_bf16(s_in, sl.CT, sl.Cb, (size_t)(j1 - j0) * d));
+    }
     return cudaEventRecord(sl.in_done, s_in);
   };
 
@@ -412,6 +418,12 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
                                                   reinterpret_cast<uintptr_t>(e.U) | reinterpret_cast<uintptr_t>(e.Mo) |
                                                   reinterpret_cast<uintptr_t>(e.Vo) | reinterpret_cast<uintptr_t>(e.Wpart)) & 15u) == 0;
     auto gemm_w = [&]() {
+      if (use_tc) {   // C (bf16 copy) x Q (bf16) on the tensor cores, split over d
+        int ns = 1;
+        (void)extend_tc_w(s_cmp, sl.mapC, &tc_maps, nc, d, k, e.Wpart, kSplitW, &ns, e.flags);
+        sum_splits_kernel<<<148 * 2, 256, 0, s_cmp>>>(e.Wpart, plane, ns, e.W);
+        return;
+      }
       if (vec) gemm_kernel<64, false, true, SplitEpi><<<gw, 256, 0, s_cmp>>>(sl.CT, d_Q, nc, k, d, kper, SplitEpi{e.Wpart, plane});
       else gemm_kernel<64, false, false, SplitEpi><<<gw, 256, 0, s_cmp>>>(sl.CT, d_Q, nc, k, d, kper, SplitEpi{e.Wpart, plane});
       sum_splits_kernel<<<148 * 2, 256, 0, s_cmp>>>(e.Wpart, plane, nsplit, e.W);
@@ -423,7 +435,7 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
       p1 *= cfg->beta1; p2 *= cfg->beta2;
       AdamArgs aa{cfg->eta, 2.f * cfg->lambda, cfg->beta1, cfg->beta2, cfg->eps, (float)(1.0 / (1.0 - p1)),
                   (float)(1.0 / (1.0 - p2))};
-      if (use_tc) CK(extend_tc_adam(s_cmp, e.U, tm_q, nc, d, k, sl.CT, e.Mo, e.Vo, aa, e.flags));
+      if (use_tc) CK(extend_tc_adam(s_cmp, e.U, &tc_maps, nc, d, k, sl.CT, e.Mo, e.Vo, sl.Cb, aa, e.flags));
       else if (vec) gemm_kernel<128, true, true, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
       else gemm_kernel<128, true, false, AdamEpi><<<ga, 256, 0, s_cmp>>>(e.U, d_Q, nc, d, k, k, AdamEpi{sl.CT, e.Mo, e.Vo, aa});
     }
@@ -445,7 +457,8 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
     return cudaEventRecord(sl.out_done, s_out);
   };
 
-  if (err == cudaSuccess && use_tc) err = extend_tc_prepare(s_cmp, d_Q, d, k, e.Qb, tm_q);
+  if (err == cudaSuccess && use_tc) err = extend_tc_prepare(s_cmp, d_Q, d, k, e.Qb, &tc_maps);
+  for (int s = 0; s < 2 && err == cudaSuccess && use_tc; ++s) err = extend_tc_map_c(e.slot[s].Cb, cc, d, e.slot[s].mapC);
   if (err == cudaSuccess) err = cudaMemsetAsync(e.flags, 0, sizeof(int32_t) * FLAG_COUNT, s_cmp);
   if (err == cudaSuccess) err = cudaMemsetAsync(e.sse, 0, sizeof(double), s_cmp);
   if (err == cudaSuccess) err = cudaStreamSynchronize(s_cmp);

@@ -29,6 +29,16 @@ namespace {
 
 #include "tc_common.cuh"
 
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 constexpr int BLK = 128;
 constexpr int NSY = 4;   // stages of the Q tile ring
 constexpr int STG_LD = 36;   // floats per staged row (32 + 4: float4-aligned, rows four banks apart)
@@ -58,8 +68,8 @@ __device__ __forceinline__ float adam_one(const AdamArgs &a, float acc, float c,
 template <int K>
 __global__ void __launch_bounds__(576, 1)
 adam_gemm_tc_kernel(const float *__restrict__ U, const __grid_constant__ CUtensorMap tmQ, int nc, int d, int nsplit,
-                    float *__restrict__ Cm, float *__restrict__ Mo, float *__restrict__ Vo, AdamArgs aa,
-                    int32_t *__restrict__ flags) {
+                    float *__restrict__ Cm, float *__restrict__ Mo, float *__restrict__ Vo,
+                    __nv_bfloat16 *__restrict__ Cb, AdamArgs aa, int32_t *__restrict__ flags) {
   using L = ESmem<K>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;
@@ -208,6 +218,12 @@ adam_gemm_tc_kernel(const float *__restrict__ U, const __grid_constant__ CUtenso
               __stcs(reinterpret_cast<float4 *>(Cm + o), c[r]);
               __stcs(reinterpret_cast<float4 *>(Mo + o), mo[r]);
               __stcs(reinterpret_cast<float4 *>(Vo + o), vo[r]);
+              // the bf16 copy the next step's first product reads
+              __nv_bfloat162 lo = __floats2bfloat162_rn(c[r].x, c[r].y), hi = __floats2bfloat162_rn(c[r].z, c[r].w);
+              uint2 pk;
+              pk.x = *reinterpret_cast<uint32_t *>(&lo);
+              pk.y = *reinterpret_cast<uint32_t *>(&hi);
+              __stcs(reinterpret_cast<uint2 *>(Cb + o), pk);
             }
           }
         }
@@ -224,6 +240,121 @@ adam_gemm_tc_kernel(const float *__restrict__ U, const __grid_constant__ CUtenso
   }
 }
 
+// ---- first product of a step: W = C Q (chunk columns x rank, contraction over the d template columns) --
+// CTA = 128 rows of the chunk x one slice of d (split-K; the partial planes are added in split order by
+// the caller).  Per 64 template columns: the C tile (128 x 64 bf16, K-major) and the Q tile (64 rows x
+// K rank columns, read MN-major: its rows are the contraction index) arrive by TMA; four tcgen05.mma
+// of 128 x K x 16 accumulate into one fp32 block in TMEM; after the slice, four warps store the block.
+constexpr int WST = 6;   // stages of the (C tile, Q tile) ring
+
+template <int K>
+struct WSmem {
+  static constexpr int A_BYTES = BLK * 128;        // 128 rows x 64 bf16
+  static constexpr int B_BYTES = (K / 64) * 64 * 128;   // 64 rows x K bf16, in 64-column blocks
+  static constexpr int STAGE = A_BYTES + B_BYTES;
+  static constexpr int OFF_BAR = WST * STAGE;
+  static constexpr int TOTAL = OFF_BAR + 256 + 1024;
+  static constexpr int B_FULL = 0, B_EMPTY = WST, B_DONE = 2 * WST, B_COUNT = 2 * WST + 1;
+  static_assert(B_COUNT * 8 <= 192, "barriers overlap the TMEM address slot");
+};
+
+template <int K>
+__global__ void __launch_bounds__(192, 1)
+w_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmQ64, int nc, int d,
+                 int nsplit, float *__restrict__ Wpart, size_t plane, int32_t *__restrict__ flags) {
+  using L = WSmem<K>;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char *smp = smem_dyn + (sm0 - s32(smem_dyn));
+  const uint32_t bar0 = sm0 + L::OFF_BAR;
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smp + L::OFF_BAR + 192);
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ib = blockIdx.x / nsplit, sp = blockIdx.x % nsplit;
+  const int NS = (d + 63) / 64;                                   // 64-column steps over d
+  const int s0 = (int)((long long)NS * sp / nsplit), s1 = (int)((long long)NS * (sp + 1) / nsplit);
+  const int NW = s1 - s0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < WST; ++s) { mbar_init(bar(L::B_FULL + s), 1); mbar_init(bar(L::B_EMPTY + s), 1); }
+    mbar_init(bar(L::B_DONE), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;" ::"r"(bar0 + 192u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  bool ok = true;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int w = 0; w < NW && ok; ++w) {
+        const int st = w % WST;
+        if (w >= WST) ok = mbar_wait(bar(L::B_EMPTY + st), ((w / WST) - 1) & 1);
+        if (!ok) break;
+        mbar_expect_tx(bar(L::B_FULL + st), L::STAGE);
+        const uint32_t a = sm0 + st * L::STAGE;
+        tma_load_2d(a, &tmC, bar(L::B_FULL + st), (s0 + w) * 64, ib * BLK);              // columns beyond d: zeros
+        for (int c = 0; c < K / 64; ++c)
+          tma_load_2d(a + L::A_BYTES + c * 64 * 128, &tmQ64, bar(L::B_FULL + st), c * 64, (s0 + w) * 64);   // rows beyond d: zeros
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t ID = idesc_bf16(K) | (1u << 16);   // B is MN-major
+      for (int w = 0; w < NW && ok; ++w) {
+        const int st = w % WST;
+        ok = mbar_wait(bar(L::B_FULL + st), (w / WST) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a = sm0 + st * L::STAGE, b = a + L::A_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)   // 16 template columns per step: 32 B along a C row, 16 rows (2048 B) of the Q tile
+          tc_mma_ss(tmem, smem_desc(a + ks * 32), smem_desc_mn(b + ks * 2048, 64 * 128), ID, (w > 0 || ks > 0));
+        tc_commit(bar(L::B_EMPTY + st));
+      }
+      if (ok) tc_commit(bar(L::B_DONE));
+    }
+    __syncwarp();
+  } else {
+    // ---- four warps store the accumulated block (a slice with no steps stores zeros) --------------------
+    const int q = warp & 3;
+    const int row = q * 32 + lane, gr = ib * BLK + row;
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    if (NW > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(L::B_DONE), 0));
+    if (ok) {
+      tc_fence_after();
+      float *dst = Wpart + (size_t)sp * plane + (size_t)gr * K;
+#pragma unroll
+      for (int c = 0; c < K / 32; ++c) {
+        uint32_t gv[32];
+        if (NW > 0) tc_ld32(tmem + lane_off + c * 32, gv);
+        else {
+#pragma unroll
+          for (int v = 0; v < 32; ++v) gv[v] = 0u;
+        }
+        if (gr < nc) {
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            *reinterpret_cast<uint4 *>(dst + c * 32 + v * 4) = make_uint4(gv[4 * v], gv[4 * v + 1], gv[4 * v + 2], gv[4 * v + 3]);
+        }
+      }
+    }
+  }
+  if (!ok && lane == 0) flags[FLAG_TIMEOUT] = 1;
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;" ::"r"(tmem) : "memory");
+  }
+}
+
 __global__ void to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t n) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
@@ -231,34 +362,71 @@ __global__ void to_bf16_kernel(const float *__restrict__ src, __nv_bfloat16 *__r
 
 template <int K>
 cudaError_t launch_adam_tc(cudaStream_t st, const float *U, const CUtensorMap &tmQ, int nc, int d, float *Cm, float *Mo,
-                           float *Vo, const AdamArgs &aa, int32_t *flags) {
+                           float *Vo, __nv_bfloat16 *Cb, const AdamArgs &aa, int32_t *flags) {
   auto kern = adam_gemm_tc_kernel<K>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ESmem<K>::TOTAL));
   const int nrb = (nc + BLK - 1) / BLK, nj = (d + BLK - 1) / BLK;
   int nsplit = 148 / nrb;
   if (nsplit > nj / 4) nsplit = nj / 4;
   if (nsplit < 1) nsplit = 1;
-  kern<<<nrb * nsplit, 576, ESmem<K>::TOTAL, st>>>(U, tmQ, nc, d, nsplit, Cm, Mo, Vo, aa, flags);
+  kern<<<nrb * nsplit, 576, ESmem<K>::TOTAL, st>>>(U, tmQ, nc, d, nsplit, Cm, Mo, Vo, Cb, aa, flags);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-// Whether the tensor-core form exists for this shape: rank 64 or 128, every row of C 16-byte aligned.
-bool extend_tc_qualifies(int32_t d, int32_t k) { return (k == 64 || k == 128) && d % 4 == 0 && d >= 128; }
+// Whether the tensor-core form exists for this shape: rank 64 or 128, every row of C 16-byte aligned in both
+// its fp32 and its bf16 copy.
+bool extend_tc_qualifies(int32_t d, int32_t k) { return (k == 64 || k == 128) && d % 8 == 0 && d >= 128; }
 
-// bf16 copy of Q (d x k) into `qb` and its tensor map (stored in `tm`, 128 bytes)
-cudaError_t extend_tc_prepare(cudaStream_t st, const float *d_Q, int32_t d, int32_t k, __nv_bfloat16 *qb, void *tm) {
+// Per call: the bf16 copy of Q (d x k) and its two tensor maps (128-row tiles for the gradient product,
+// 64-row tiles for the first product).  `maps` is host memory for the ExtendTcMaps of this call.
+cudaError_t extend_tc_prepare(cudaStream_t st, const float *d_Q, int32_t d, int32_t k, __nv_bfloat16 *qb, ExtendTcMaps *maps) {
   to_bf16_kernel<<<148 * 4, 256, 0, st>>>(d_Q, qb, (size_t)d * k);
   CK(cudaGetLastError());
-  return make_map(static_cast<CUtensorMap *>(tm), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, qb, (uint64_t)d, (uint64_t)k, BLK);
+  CK(make_map(reinterpret_cast<CUtensorMap *>(maps->q128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, qb, (uint64_t)d, (uint64_t)k, BLK));
+  return make_map(reinterpret_cast<CUtensorMap *>(maps->q64), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, qb, (uint64_t)d, (uint64_t)k, 64);
 }
 
-cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const void *tm, int32_t nc, int32_t d, int32_t k, float *Cm,
-                           float *Mo, float *Vo, const AdamArgs &aa, int32_t *flags) {
-  const CUtensorMap &tmQ = *static_cast<const CUtensorMap *>(tm);
-  if (k == 128) return launch_adam_tc<128>(st, U, tmQ, nc, d, Cm, Mo, Vo, aa, flags);
-  return launch_adam_tc<64>(st, U, tmQ, nc, d, Cm, Mo, Vo, aa, flags);
+// Per slot: the tensor map of the bf16 coefficient buffer (rows = chunk capacity, d columns).
+cudaError_t extend_tc_map_c(__nv_bfloat16 *cb, int32_t rows, int32_t d, void *map) {
+  return make_map(static_cast<CUtensorMap *>(map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, cb, (uint64_t)rows, (uint64_t)d, BLK);
+}
+
+cudaError_t extend_tc_to_bf16(cudaStream_t st, const float *src, __nv_bfloat16 *dst, size_t n) {
+  to_bf16_kernel<<<148 * 4, 256, 0, st>>>(src, dst, n);
+  return cudaGetLastError();
+}
+
+// W partial planes [nsplit][nc x k] = C Q over the slices of d; returns the number of planes in *nsplit_out.
+cudaError_t extend_tc_w(cudaStream_t st, const void *map_c, const ExtendTcMaps *maps, int32_t nc, int32_t d, int32_t k,
+                        float *Wpart, int max_split, int *nsplit_out, int32_t *flags) {
+  const int nrb = (nc + BLK - 1) / BLK, ns = (d + 63) / 64;
+  int nsplit = 148 / nrb;
+  if (nsplit > max_split) nsplit = max_split;
+  if (nsplit > ns) nsplit = ns;
+  if (nsplit < 1) nsplit = 1;
+  *nsplit_out = nsplit;
+  const CUtensorMap &tmC = *static_cast<const CUtensorMap *>(map_c);
+  const CUtensorMap &tmQ = *reinterpret_cast<const CUtensorMap *>(maps->q64);
+  const size_t plane = (size_t)nc * k;
+  if (k == 128) {
+    auto kern = w_gemm_tc_kernel<128>;
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WSmem<128>::TOTAL));
+    kern<<<nrb * nsplit, 192, WSmem<128>::TOTAL, st>>>(tmC, tmQ, nc, d, nsplit, Wpart, plane, flags);
+  } else {
+    auto kern = w_gemm_tc_kernel<64>;
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WSmem<64>::TOTAL));
+    kern<<<nrb * nsplit, 192, WSmem<64>::TOTAL, st>>>(tmC, tmQ, nc, d, nsplit, Wpart, plane, flags);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const ExtendTcMaps *maps, int32_t nc, int32_t d, int32_t k,
+                           float *Cm, float *Mo, float *Vo, __nv_bfloat16 *Cb, const AdamArgs &aa, int32_t *flags) {
+  const CUtensorMap &tmQ = *reinterpret_cast<const CUtensorMap *>(maps->q128);
+  if (k == 128) return launch_adam_tc<128>(st, U, tmQ, nc, d, Cm, Mo, Vo, Cb, aa, flags);
+  return launch_adam_tc<64>(st, U, tmQ, nc, d, Cm, Mo, Vo, Cb, aa, flags);
 }
 
 }  // namespace tsid

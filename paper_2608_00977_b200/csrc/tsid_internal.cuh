@@ -131,10 +131,18 @@ cudaError_t scan_u32(const uint32_t *in, uint32_t *out, int64_t n, LayoutScratch
 struct AdamArgs {
   float lr, lam2, b1, b2, eps, c1, c2;   // c1 = 1/(1-b1^t), c2 = 1/(1-b2^t)
 };
+struct ExtendTcMaps {                       // host copies of the tensor maps of the bf16 Q (128 bytes each)
+  alignas(64) unsigned char q128[128];
+  alignas(64) unsigned char q64[128];
+};
 bool extend_tc_qualifies(int32_t d, int32_t k);
-cudaError_t extend_tc_prepare(cudaStream_t st, const float *d_Q, int32_t d, int32_t k, __nv_bfloat16 *qb, void *tm);
-cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const void *tm, int32_t nc, int32_t d, int32_t k, float *Cm,
-                           float *Mo, float *Vo, const AdamArgs &aa, int32_t *flags);
+cudaError_t extend_tc_prepare(cudaStream_t st, const float *d_Q, int32_t d, int32_t k, __nv_bfloat16 *qb, ExtendTcMaps *maps);
+cudaError_t extend_tc_map_c(__nv_bfloat16 *cb, int32_t rows, int32_t d, void *map);
+cudaError_t extend_tc_to_bf16(cudaStream_t st, const float *src, __nv_bfloat16 *dst, size_t n);
+cudaError_t extend_tc_w(cudaStream_t st, const void *map_c, const ExtendTcMaps *maps, int32_t nc, int32_t d, int32_t k,
+                        float *Wpart, int max_split, int *nsplit_out, int32_t *flags);
+cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const ExtendTcMaps *maps, int32_t nc, int32_t d, int32_t k,
+                           float *Cm, float *Mo, float *Vo, __nv_bfloat16 *Cb, const AdamArgs &aa, int32_t *flags);
 
 // sparse passes (sparse.cu)
 cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);

@@ -84,8 +84,8 @@ def test_extend_errors():
     assert B.lib().tsid_extend_workspace_bytes(C.byref(cfg), torch.tensor(cp).data_ptr(), C.byref(need)) == B.TSID_ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("m,d,k,ncols,per_col,chunk", [(800, 200, 64, 257, 80, 100), (600, 260, 128, 300, 70, 150),
-                                                       (900, 1028, 64, 700, 90, 333)])
+@pytest.mark.parametrize("m,d,k,ncols,per_col,chunk", [(800, 200, 64, 257, 80, 100), (600, 264, 128, 300, 70, 150),
+                                                       (900, 1032, 64, 700, 90, 333)])
 def test_extend_tensor_core_form(m, d, k, ncols, per_col, chunk):
     """TSID_EXTEND_TC: the gradient product on the tensor cores with bf16 operands (the paper's mixed
     precision).  Adam turns a gradient coordinate into a step of about +-eta whatever its size, so where the
@@ -100,6 +100,14 @@ def test_extend_tensor_core_form(m, d, k, ncols, per_col, chunk):
     B.tsid_extend(*args, Ch, chunk, 1, 1.0, 0.05, eps=1e4, tensor_cores=True)
     Cr, _ = oracle.extend(m, d, k, cp, ri, v, P, Q, 1.0, 0.05, 1, eps=1e4)
     assert relerr(Ch.numpy(), Cr) <= 1e-2, relerr(Ch.numpy(), Cr)       # bf16 operands, fp32 accumulation
+    # (1b) the same from random coefficients (warm start): the step now also depends on the first product W = C Q
+    rng = np.random.default_rng(5)
+    C0 = (rng.standard_normal((ncols, d)) * 0.05).astype(np.float32)
+    Ch.copy_(torch.tensor(C0))
+    B.tsid_extend(*args, Ch, chunk, 1, 1.0, 0.05, eps=1e4, tensor_cores=True)
+    Cr, _ = oracle.extend(m, d, k, cp, ri, v, P, Q, 1.0, 0.05, 1, C0=C0, eps=1e4)
+    step_err = float(np.max(np.abs((Ch.numpy() - C0) - (Cr - C0))) / np.max(np.abs(Cr - C0)))
+    assert step_err <= 1e-2, step_err
     # (2) the fit
     eta, lam, iters = 0.02, 0.05, 12
     Ch.zero_()
