@@ -156,7 +156,16 @@ rs_scatter_kernel(SortIO<NP> io, int64_t n, int64_t per_block, int shift, uint32
     for (int it = 0; it < RS_ITEMS; ++it) {
       const bool ok = wbase + it * 32 + lane < hi;
       const uint32_t dig = ok ? ((key[it] >> shift) & mask) : 0xffffffffu;
-      uint32_t peers = __match_any_sync(0xffffffffu, dig);
+      // lanes with the same digit, from one ballot per digit bit (the match instruction takes time in
+      // proportion to the number of distinct values in the warp, which is ~28 for a 7-bit digit)
+      uint32_t peers = __ballot_sync(0xffffffffu, ok);
+      if (!ok) peers = ~peers;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        if ((mask >> b) == 0) break;
+        const uint32_t bal = __ballot_sync(0xffffffffu, (dig >> b) & 1u);
+        peers &= ((dig >> b) & 1u) ? bal : ~bal;
+      }
       int leader = __ffs(peers) - 1;
       uint32_t base = 0;
       if (lane == leader && ok) {
