@@ -258,10 +258,12 @@ tsid_status_t tsid_sample_template(int32_t m, int32_t n, int64_t nnz, double alp
  *     (zeros for a cold start) and overwritten with the result.
  *   - h_sse_or_null: HOST, receives sum_Omega e^2 at the returned coefficients.
  *   - cfg.workspace: DEVICE, tsid_extend_workspace_bytes(cfg, h_col_ptr) bytes (it depends on the
- *     largest chunk); nothing is allocated on the device.  The call creates two helper streams and a
- *     few events, and synchronises before it returns.
+ *     largest chunk); nothing is allocated on the device.  The call creates two helper streams, a few
+ *     events and 64 bytes of pinned host memory (released before it returns), and synchronises before
+ *     it returns.
  * Limits: k a multiple of 4 in [4, 128]; at most 2^31 - 3 entries per chunk.  Errors: INVALID_ARG,
- * UNSUPPORTED (k), OOM (workspace), INDEX_RANGE (a row index outside [0, m)), CUDA. */
+ * UNSUPPORTED (k, or a shape TSID_EXTEND_TC does not take), OOM (workspace), INDEX_RANGE (a row index
+ * outside [0, m)), CUDA (also when a bounded device-side wait of the tensor-core kernels expired). */
 enum {
   TSID_EXTEND_COLD_START = 1u,   /* start from C = 0, h_C is only written */
   TSID_EXTEND_TC = 2u            /* mixed precision as in the paper's Stage II (Sec. 5.2): both products of a
@@ -276,7 +278,7 @@ typedef struct {
   int32_t chunk_cols;  /* chunk width (Delta c)                                         */
   int32_t iters;       /* Adam steps per chunk                                          */
   float eta, lambda, beta1, beta2, eps;
-  uint32_t flags;      /* TSID_EXTEND_COLD_START: start from C = 0, h_C is only written */
+  uint32_t flags;      /* TSID_EXTEND_COLD_START | TSID_EXTEND_TC (above)                */
   void *stream;           /* compute stream (cudaStream_t) owned by the caller          */
   void *workspace;        /* DEVICE memory owned by the caller, 256-byte aligned        */
   size_t workspace_bytes;
