@@ -410,14 +410,31 @@ tsid_status_t tsid_fit_host(const tsid_config_t *cfg, const int32_t *h_rows, con
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_cols, h_cols, nnz * 4, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_vals, h_vals, nnz * 4, cudaMemcpyHostToDevice, s);
   }
-  if (e == cudaSuccess) e = cudaMemcpyAsync(d_P, h_P, pb, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(d_Q, h_Q, qb, cudaMemcpyHostToDevice, s);
-  if (e != cudaSuccess) return cuda_fail(nullptr, e);
+  // The factors travel on a second stream, behind the triples on the bus but beside the layout pass on
+  // the device: the layout only needs the triples.
+  cudaStream_t s2 = nullptr;
+  cudaEvent_t coo_in = nullptr, fac_in = nullptr;
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&coo_in, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&fac_in, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventRecord(coo_in, s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(s2, coo_in, 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_P, h_P, pb, cudaMemcpyHostToDevice, s2);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_Q, h_Q, qb, cudaMemcpyHostToDevice, s2);
+  if (e == cudaSuccess) e = cudaEventRecord(fac_in, s2);
+  auto release = [&]() {
+    if (s2) { cudaStreamSynchronize(s2); cudaStreamDestroy(s2); }
+    if (coo_in) cudaEventDestroy(coo_in);
+    if (fac_in) cudaEventDestroy(fac_in);
+  };
+  if (e != cudaSuccess) { release(); return cuda_fail(nullptr, e); }
   tsid_config_t c2 = *cfg;
   c2.workspace_bytes = base;
   tsid_template *t = nullptr;
   st = tsid_template_create(&c2, d_rows, d_cols, d_vals, &t);
-  if (st != TSID_OK) return st;
+  if (st != TSID_OK) { release(); return st; }
+  e = cudaStreamWaitEvent(s, fac_in, 0);
+  if (e != cudaSuccess) { release(); tsid_destroy(t); return cuda_fail(nullptr, e); }
   st = tsid_fit(t, d_P, d_Q, epochs, 0, nullptr);
   if (st == TSID_OK && h_sse_or_null) st = tsid_loss(t, d_P, d_Q, h_sse_or_null, nullptr);
   if (st == TSID_OK) {
@@ -428,6 +445,7 @@ tsid_status_t tsid_fit_host(const tsid_config_t *cfg, const int32_t *h_rows, con
   }
   if (st != TSID_OK) snprintf(g_create_err, 256, "%s", t->err);
   tsid_destroy(t);
+  release();
   return st;
 }
 

@@ -245,3 +245,26 @@ def test_byte_value_streams_give_the_same_bits(precision, k):
     with pytest.raises(B.TsidError) as e:
         B.Template(B.make_config(w.m, w.n, w.k, tpl.nnz, flags=B.TSID_VALUES_U8), tpl.rows, tpl.cols, bad)
     assert e.value.status == B.TSID_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("precision", ["f32", "bf16"])
+def test_host_buffer_call_equals_the_device_path(precision):
+    """tsid_fit_host (pinned host triples and factors in, fitted factors out; the factors are uploaded on a
+    second stream while the layout is built) gives bitwise what create + fit give on device buffers."""
+    w = small_workload("host", 2100, 1300, 32, 150_000, positions="zipf", precision=precision, seed=77,
+                       values="ratings", eta=0.05, lam=0.03, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT,
+                       norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    T = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    P, Q = tpl.P0.clone(), tpl.Q0.clone()
+    T.tsid_fit(P, Q, 4)
+    sse_dev, _ = T.tsid_loss(P, Q)
+    T.tsid_destroy()
+    prec = B.TSID_BF16_SHADOW if precision == "bf16" else B.TSID_F32
+    cfg = B.make_config(w.m, w.n, w.k, tpl.nnz, prec, B.TSID_PATH_SPARSE, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
+    ws = torch.empty(B.tsid_workspace_bytes_host(cfg) + 256, dtype=torch.uint8, device=DEV)
+    hP, hQ = tpl.P0.cpu().pin_memory(), tpl.Q0.cpu().pin_memory()
+    sse = B.tsid_fit_host(cfg, tpl.rows.cpu().pin_memory(), tpl.cols.cpu().pin_memory(), tpl.vals.cpu().pin_memory(),
+                          hP, hQ, 4, ws, want_sse=True)
+    assert torch.equal(hP, P.cpu()) and torch.equal(hQ, Q.cpu())
+    assert sse == sse_dev
