@@ -272,9 +272,9 @@ class Template:
             self._raise(st)
         return n.value, a.value, b.value, c.value
 
-    def tsid_get_layout(self):
-        """Copies of the layout arrays as torch tensors (row_ptr, col_idx, val_csr, col_ptr, row_idx,
-        val_csc, perm)."""
+    def tsid_get_layout(self, copy=True):
+        """The layout arrays as torch tensors (row_ptr, col_idx, val_csr, col_ptr, row_idx, val_csc, perm):
+        copies, or with copy=False views into the workspace that die with the template."""
         ptrs = [C.c_void_p(None) for _ in range(7)]
         st = lib().tsid_get_layout(self.h, *[C.byref(p) for p in ptrs])
         if st != TSID_OK:
@@ -288,7 +288,8 @@ class Template:
         for p, (dt, cnt) in zip(ptrs, spec):
             off = p.value - base + (base - self.workspace.data_ptr())
             nbytes = cnt * torch.empty(0, dtype=dt).element_size()
-            out.append(self.workspace[off:off + nbytes].view(dt).clone())
+            v = self.workspace[off:off + nbytes].view(dt)
+            out.append(v.clone() if copy else v)
         return out
 
     def tsid_destroy(self):
