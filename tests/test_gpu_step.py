@@ -99,6 +99,34 @@ def test_split_rows_and_empty_rows():
         T.tsid_destroy()
 
 
+@pytest.mark.parametrize("precision,emu", [(B.TSID_F32, False), (B.TSID_BF16_SHADOW, True)])
+def test_degenerate_shapes(precision, emu):
+    """One cell, one row, one column, and a fully observed matrix (Omega = every cell)."""
+    rng = np.random.default_rng(17)
+    k = 16
+    for m, n in ((1, 1), (1, 3000), (3000, 1), (37, 53)):
+        ids = np.arange(m * n)
+        rows, cols = (ids // n).astype(np.int32), (ids % n).astype(np.int32)
+        p = rng.permutation(m * n); rows, cols = rows[p], cols[p]
+        vals = rng.standard_normal(m * n).astype(np.float32)
+        P0 = (rng.standard_normal((m, k)) * 0.5).astype(np.float32); Q0 = (rng.standard_normal((n, k)) * 0.5).astype(np.float32)
+        cfg = B.make_config(m, n, k, m * n, precision, B.TSID_PATH_SPARSE, 0.05, 0.03, 0.1, B.TSID_CLIP_ASYM_STEP, 1, 1,
+                            B.TSID_VALIDATE)
+        T = B.Template(cfg, torch.tensor(rows, device=DEV), torch.tensor(cols, device=DEV), torch.tensor(vals, device=DEV))
+        P = torch.tensor(P0, device=DEV); Q = torch.tensor(Q0, device=DEV)
+        GP, GQ = torch.empty_like(P), torch.empty_like(Q)
+        T.tsid_grad_step(P, Q, GP, GQ)
+        T.tsid_check()
+        ref = oracle.grad_step(m, n, k, rows, cols, vals, P0, Q0, 0.05, 0.03, 0.1, 1, 1, 1, bf16_emulate=emu)
+        for got, want in ((GP, ref.GP), (GQ, ref.GQ), (P, ref.P), (Q, ref.Q)):
+            assert relerr(got.cpu().numpy(), want) <= F32_TOL, (m, n)
+        if not emu:   # the fully observed case is the textbook dense formula
+            E = np.zeros((m, n)); E[rows, cols] = vals
+            E = E - P0.astype(np.float64) @ Q0.astype(np.float64).T
+            assert relerr(GP.cpu().numpy(), E @ Q0) <= F32_TOL and relerr(GQ.cpu().numpy(), E.T @ P0) <= F32_TOL
+        T.tsid_destroy()
+
+
 def test_zero_gradient_at_truth_and_empty_template():
     m, n, k = 300, 200, 16
     rng = np.random.default_rng(4)
