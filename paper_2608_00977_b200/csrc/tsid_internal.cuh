@@ -79,6 +79,13 @@ struct tsid_template {
   int32_t *flags;     // device flags: [0] range, [1] unsorted, [2] duplicate, [3] non-finite
   tsid::DenseState *dense;
   tsid::Prof prof;
+  // tsid_fit replays its epochs from an executable graph: fit_steps steps on the factor arrays
+  // fit_P / fit_Q, captured on fit_cap (no work ever runs there) and kept until arrays or count change
+  cudaGraphExec_t fit_exec;
+  cudaStream_t fit_cap;
+  const float *fit_P, *fit_Q;
+  int fit_steps;
+  bool fit_graph_off;  // a capture failed once: launch step by step from then on
   char err[256];
 };
 

@@ -202,6 +202,33 @@ def test_c1_fit_trajectory_and_loss():
     assert torch.equal(P3, P) and torch.equal(Q3, Q)
 
 
+@pytest.mark.parametrize("path,precision", [(B.TSID_PATH_SPARSE, B.TSID_F32), (B.TSID_PATH_SPARSE, B.TSID_BF16_SHADOW),
+                                            (B.TSID_PATH_DENSE_TC, B.TSID_BF16_SHADOW)])
+def test_fit_graph_replay_equals_step_by_step(path, precision):
+    """tsid_fit replays its epochs from a captured graph (8 steps per launch, the rest one by one): bitwise the
+    factors of the same number of tsid_grad_step calls; again on the same arrays (the cached graph), on other
+    arrays (a new capture) and below the replay threshold."""
+    w = small_workload("graph", 512, 384, 64, 30_000, positions="zipf", seed=21, values="ratings", noise_var=0.25,
+                       eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT, norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    T = B.template_from_workload(tpl, path=path, precision=precision)
+    assert T.tsid_get_info()[0] == path
+    Pa, Qa = tpl.P0.clone(), tpl.Q0.clone()
+    Pb, Qb = tpl.P0.clone(), tpl.Q0.clone()
+    Pr, Qr = tpl.P0.clone(), tpl.Q0.clone()
+    done = 0
+    for epochs, (P, Q) in ((37, (Pa, Qa)), (16, (Pa, Qa)), (5, (Pa, Qa)), (58, (Pb, Qb))):
+        if P is Pb:
+            Pr.copy_(tpl.P0); Qr.copy_(tpl.Q0)
+        T.tsid_fit(P, Q, epochs)
+        for _ in range(epochs):
+            T.tsid_grad_step(Pr, Qr)
+        T.tsid_check()
+        assert torch.equal(P, Pr) and torch.equal(Q, Qr), (epochs, done)
+        done += epochs
+    T.tsid_destroy()
+
+
 def test_objective_with_regulariser():
     w = small_workload("obj", 800, 600, 32, 40_000, seed=11, lam=0.05)
     tpl = W.make_template(w, DEV, order="shuffled")
