@@ -568,7 +568,7 @@ def main():
                     "pass_R": {"ms": row_ms / max(1, nrec)}, "pass_RT": {"ms": col_ms / max(1, nrec)},
                     "update": {"ms": upd_ms / max(1, nrec)},
                     "step_frac": 6.0 * w.m * w.n * w.k / (ms / args.steps * 1e-3) / 1e12 / tf_sustained,
-                    "frac_of_nominal_2250": tfl / 2250.0}
+                    "frac_of_burst": tfl / tf_burst, "frac_of_nominal_2250": tfl / 2250.0}
 
     roofline.update(timing_note)
 
