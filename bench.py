@@ -552,6 +552,12 @@ def main():
                 "step_compulsory_bytes": nnz * 16 + (w.m + w.n) * w.k * 20,   # perfect cache: streams + factors once
                 "step_frac": (b_row + b_col + b_upd) / (ms / args.steps * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+    tr = NCU_TRAFFIC_PER_LAUNCH.get(args.workload)
+    if tr and pass_ms > 0:
+        # what HBM itself carried (ncu's DRAM bytes of a launch over this run's launch time): the algorithmic
+        # figure above counts every gathered row as if it came from HBM, and L2 serves most of them
+        roofline["dram_gbs"] = tr / (pass_ms * 1e-3) / 1e9
+        roofline["dram_frac"] = roofline["dram_gbs"] / peak
     timing_note = {"launch_times_from": "the same %d steps repeated with the library's per-kernel CUDA events" % args.steps,
                    "ms_per_step_with_events": ms_profiled / args.steps}
     if path == B.TSID_PATH_DENSE_TC:
