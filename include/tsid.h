@@ -178,7 +178,8 @@ tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or
  * whole call when epochs <= 16, else 8 steps per launch and the rest step by step): captured once on
  * a stream of the library's own, launched into cfg.stream, kept with the template while d_P, d_Q and
  * the step count stay the same.  The results are bitwise those of the same number of tsid_grad_step
- * calls.  If the capture fails, the steps launch one by one, in this and every later call. */
+ * calls.  If the capture fails, the steps launch one by one, in this and every later call; they also do
+ * while cfg.stream is itself being captured by the caller (the call can be part of a caller's graph). */
 tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epochs,
                        int32_t loss_every, double *h_sse_history_or_null);
 

@@ -323,7 +323,14 @@ tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epoch
   }
   cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
   int ep = 0;
-  if (e == cudaSuccess && loss_every == 0 && !t->prof.on && !t->fit_graph_off && epochs >= kFitGraphMin) {
+  // a caller that is capturing cfg.stream into a graph of its own gets plain launches
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (e == cudaSuccess && cudaStreamIsCapturing(t->stream, &capturing) != cudaSuccess) {
+    cudaGetLastError();
+    capturing = cudaStreamCaptureStatusActive;
+  }
+  if (e == cudaSuccess && loss_every == 0 && !t->prof.on && !t->fit_graph_off && epochs >= kFitGraphMin &&
+      capturing == cudaStreamCaptureStatusNone) {
     const int per = epochs <= kFitGraphMax ? epochs : kFitGraphEpochs;
     if (fit_graph_get(t, d_P, d_Q, per) == cudaSuccess) {
       for (; ep + per <= epochs && e == cudaSuccess; ep += per) e = cudaGraphLaunch(t->fit_exec, t->stream);

@@ -229,6 +229,34 @@ def test_fit_graph_replay_equals_step_by_step(path, precision):
     T.tsid_destroy()
 
 
+def test_fit_inside_a_callers_graph_capture():
+    """tsid_fit with loss_every = 0 enqueues work only: a caller can capture it into a CUDA graph of its own
+    (the library then launches step by step instead of replaying its own graph) and replay it."""
+    w = small_workload("cap", 384, 256, 32, 20_000, positions="zipf", seed=23, values="ratings", noise_var=0.25,
+                       eta=0.05, lam=0.03, xi=0.1, clip=W.CLIP_ASYM_STEP, norm_p=W.NORM_COUNT, norm_q=W.NORM_COUNT)
+    tpl = W.make_template(w, DEV, order="shuffled")
+    s = torch.cuda.Stream(device=DEV)
+    cfg = B.make_config(w.m, w.n, w.k, tpl.nnz, B.TSID_BF16_SHADOW, B.TSID_PATH_SPARSE, w.eta, w.lam, w.xi, w.clip,
+                        w.norm_p, w.norm_q)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        T = B.Template(cfg, tpl.rows, tpl.cols, tpl.vals, stream=s)
+        P, Q = tpl.P0.clone(), tpl.Q0.clone()
+        Pr, Qr = tpl.P0.clone(), tpl.Q0.clone()
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            T.tsid_fit(P, Q, 12)
+        g.replay()
+        g.replay()
+        for _ in range(24):
+            T.tsid_grad_step(Pr, Qr)
+        T.tsid_check()
+    torch.cuda.synchronize()
+    assert torch.equal(P, Pr) and torch.equal(Q, Qr)
+    T.tsid_destroy()
+
+
 def test_objective_with_regulariser():
     w = small_workload("obj", 800, 600, 32, 40_000, seed=11, lam=0.05)
     tpl = W.make_template(w, DEV, order="shuffled")
