@@ -261,7 +261,7 @@ update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int
 // added in rank order, the update is applied once, and the new values are stored with plain stores into
 // every rank's replica of Q: a reduce-scatter and an all-gather folded into the update, with no
 // intermediate buffer.  Since one rank computes a row and all receive the same bits, the replicas cannot
-// drift.  (No multicast and no waiting inside the kernel: the ranks synchronise before and after it.)
+// drift.  (Nothing waits inside the kernel: the ranks synchronise before and after it.)
 constexpr int kMaxPeers = 16;
 struct PeerPtrs {
   const float *gq[kMaxPeers];
