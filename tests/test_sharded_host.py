@@ -69,3 +69,14 @@ def test_no_process_group_is_identity():
     t = torch.tensor([1.0, 2.0])
     assert S.all_reduce_sum(t).tolist() == [1.0, 2.0]
     assert S.all_reduce_sum(t, dist).tolist() == [1.0, 2.0]     # module given, group not initialised
+
+
+def test_minibatch_split_is_a_seeded_partition():
+    from paper_2608_00977_b200.minibatch import split_batches
+    a = split_batches(1003, 7, 5, "cpu")
+    b = split_batches(1003, 7, 5, "cpu")
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+    assert sorted(torch.cat(a).tolist()) == list(range(1003))
+    assert max(len(x) for x in a) - min(len(x) for x in a) <= 1
+    assert not torch.equal(torch.cat(a), torch.cat(split_batches(1003, 7, 6, "cpu")))
+    assert len(split_batches(10, 1, 0, "cpu")) == 1 and len(split_batches(0, 3, 0, "cpu")) == 3
