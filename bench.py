@@ -433,13 +433,13 @@ def main():
     if rank == 0:
         G.build()
     dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
-    B.lib()
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    B.lib()
 
     w = W.CONFIGS[args.workload]
     t0 = time.perf_counter()
