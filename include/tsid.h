@@ -84,7 +84,8 @@ typedef enum { TSID_PATH_AUTO = 0, TSID_PATH_SPARSE = 1, TSID_PATH_DENSE_TC = 2 
  * contributions of a factor row are added, divided by s (Eq. 9's 1/n) and applied with eta.
  * In this mode the regulariser sits inside every entry's term, a row without entries does not
  * move, the values read are those of the template's precision, and d_gradP / d_gradQ receive
- * the sums of the c_ij.  Sparse path only. */
+ * the sums of the c_ij.  Sparse path only, and with TSID_F32 factors k <= 128 (TSID_ERR_UNSUPPORTED
+ * otherwise, from tsid_workspace_bytes and tsid_template_create). */
 typedef enum {
   TSID_CLIP_NONE = 0, TSID_CLIP_ASYM_STEP = 1, TSID_CLIP_ASYM_GRAD = 2, TSID_CLIP_ASYM_ENTRY = 3
 } tsid_clip_t;
