@@ -532,8 +532,8 @@ def main():
 
     # ---- roofline of the dominant kernel (the gather-reduce pass: two launches per step) ----------
     peak, tf_sustained, tf_burst, peak_kind = load_peaks()
-    nseg_row = w.m + nnz // 1024
-    nseg_col = w.n + nnz // 1024
+    nseg_row = w.m + nnz // 512
+    nseg_col = w.n + nnz // 512
     b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col, 1 if args.values == "u8" else 4)
     pass_ms = (row_ms + col_ms) / max(1, 2 * nrec)
     bytes_per_launch = (b_row + b_col) / 2
