@@ -33,7 +33,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the gather-reduce pass kernel
 # (average of the row pass and the column pass), from the ncu summaries under profiles/.
 NCU_TRAFFIC_PER_LAUNCH = {
-    "C5": 92.14e9,        # profiles/step_kernels_C5_launches_dram.md: row 77.23 GB, column 107.06 GB
+    "C5": 93.79e9,        # profiles/step_kernels_C5_launches_dram.md: row 78.88 GB, column 108.69 GB
     "C3": 0.865e9,        # profiles/pass_staged_kernel_C3_ncu.md
     "C4-dense": 0.551e9,  # profiles/dense_pass_kernel_C4_ncu.md: the fp16 R matrix once per launch
 }
