@@ -44,7 +44,10 @@
  * clip, and the layout against numpy.lexsort).  The bf16 path has no exact pin
  * beyond the emulation switch (inputs rounded to bf16, round-to-nearest-even):
  * the rounding function itself is pinned against a table of hand-derived bit
- * patterns.
+ * patterns, and what the switch rounds is pinned in both branches: the aggregated
+ * modes against the plain oracle on pre-rounded inputs (regulariser on the fp32
+ * master), the entry-wise clip by a hand-worked value and the same identity
+ * (there the regulariser sits inside each entry's term and reads the rounded value).
  */
 #include <math.h>
 #include <stdint.h>

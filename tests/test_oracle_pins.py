@@ -106,6 +106,41 @@ def test_worked_example_entrywise_clip(golden_3x2):
     np.testing.assert_allclose(big.DP, ref.DP, rtol=1e-15) and np.testing.assert_allclose(big.DQ, ref.DQ, rtol=1e-15)
 
 
+def test_worked_example_entrywise_clip_with_bf16_emulation(golden_3x2):
+    """The entry-wise clip on a bf16 template: rounded values wherever a factor is read (regulariser included),
+    step added to the fp32 master.  Hand-worked numbers, plus the identity with the plain branch on pre-rounded
+    factors, so that rounding only one operand, or reading the master in the regulariser, fails here."""
+    g = golden_3x2
+    m, n, k, rows, cols, vals, _, Q = _inst(g)
+    P = _arr(g, "P_emu", (m, k), np.float32)
+    eta, lam, xi = g["eta"][0], g["lambda"][0], g["xi"][0]
+    st = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, eta, lam, xi, oracle.CLIP_ASYM_ENTRY, 0, 0, bf16_emulate=True)
+    assert np.array_equal(st.GP, _arr(g, "GP_entry_emu", (m, k)))
+    assert np.array_equal(st.GQ, _arr(g, "GQ_entry_emu", (n, k)))
+    np.testing.assert_allclose(st.P, _arr(g, "P1_entry_emu_none", (m, k)), rtol=0, atol=1e-7)
+    np.testing.assert_allclose(st.Q, _arr(g, "Q1_entry_emu_none", (n, k)), rtol=0, atol=1e-7)
+    assert st.GP[0, 0] != 0.8388671875          # what the master value in the regulariser would give
+    # on random factors: the sums equal those of the plain branch fed pre-rounded factors, the step starts
+    # from the unrounded master
+    rng = np.random.default_rng(5)
+    m2, n2, k2, nnz = 23, 17, 8, 140
+    cells = rng.choice(m2 * n2, nnz, replace=False)
+    r2, c2 = (cells // n2).astype(np.int32), (cells % n2).astype(np.int32)
+    v2 = rng.normal(size=nnz).astype(np.float32)
+    P2 = rng.normal(size=(m2, k2)).astype(np.float32); Q2 = rng.normal(size=(n2, k2)).astype(np.float32)
+    rnd = np.vectorize(oracle.bf16_round, otypes=[np.float32])
+    Pr, Qr = rnd(P2), rnd(Q2)
+    assert np.any(Pr != P2) and np.any(Qr != Q2)
+    for norms in ((0, 0), (0, 1), (1, 1)):
+        emu = oracle.grad_step(m2, n2, k2, r2, c2, v2, P2, Q2, 0.05, 0.3, 0.4, oracle.CLIP_ASYM_ENTRY, *norms, bf16_emulate=True)
+        pre = oracle.grad_step(m2, n2, k2, r2, c2, v2, Pr, Qr, 0.05, 0.3, 0.4, oracle.CLIP_ASYM_ENTRY, *norms)
+        assert np.array_equal(emu.GP, pre.GP) and np.array_equal(emu.GQ, pre.GQ)
+        assert np.array_equal(emu.DP, pre.DP) and np.array_equal(emu.DQ, pre.DQ)
+        np.testing.assert_allclose(emu.P, (P2.astype(np.float64) + 0.05 * pre.DP).astype(np.float32), rtol=0, atol=0)
+        np.testing.assert_allclose(emu.Q, (Q2.astype(np.float64) + 0.05 * pre.DQ).astype(np.float32), rtol=0, atol=0)
+        assert np.any(emu.P != pre.P)
+
+
 def test_worked_example_layout(golden_3x2):
     g = golden_3x2
     lay = oracle.layout(3, 2, _arr(g, "shuf_rows", dtype=np.int32), _arr(g, "shuf_cols", dtype=np.int32),
