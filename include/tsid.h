@@ -73,8 +73,19 @@ typedef enum { TSID_F32 = 0, TSID_BF16_SHADOW = 1 } tsid_precision_t;
  * TSID_PATH_DENSE_TC: tcgen05 masked-GEMM variant (Sec. 5.1, "Regularizing Sparse RMF
  * Updates for Tensor Cores"): P Q^T, then E Q and E^T P with bf16 operands and fp32
  * accumulation; requires TSID_BF16_SHADOW, k a multiple of 16 and m, n multiples of 128.
- * TSID_PATH_AUTO picks DENSE_TC when the template qualifies and nnz / (m n) >= 0.05. */
-typedef enum { TSID_PATH_AUTO = 0, TSID_PATH_SPARSE = 1, TSID_PATH_DENSE_TC = 2 } tsid_path_t;
+ * TSID_PATH_HYBRID: both, each where it fits.  Under skewed popularity the observed cells crowd into
+ * nearly full blocks once rows and columns are ordered by their number of entries.  At create the rows and
+ * columns are ranked by degree (ties by index), the template is cut into 128 x 128 tiles in that order,
+ * and every tile with at least ~3 % of its cells observed (480 entries; more if the tiles would not fit
+ * the 16 bytes per entry of workspace reserved for them) is kept as a dense fp16 block and goes through
+ * the tensor-core pass; every other entry goes through the gather-reduce passes on a CSR / CSC of the
+ * remainder; the two partial sums of a factor row are added in a fixed order.  Needs TSID_BF16_SHADOW,
+ * k in {64, 128}, no entry-wise clip, no TSID_VALUES_U8, and nnz >= max(m, n, ceil(m/128) ceil(n/128)).
+ * If no tile reaches the threshold, if Omega holds a duplicate, or if a value in a stored tile is beyond
+ * the fp16 range, the handle runs TSID_PATH_SPARSE instead (tsid_get_info tells).
+ * TSID_PATH_AUTO picks DENSE_TC when the template qualifies and nnz / (m n) >= 0.05, else HYBRID when
+ * it qualifies and nnz >= 4,000,000, else SPARSE. */
+typedef enum { TSID_PATH_AUTO = 0, TSID_PATH_SPARSE = 1, TSID_PATH_DENSE_TC = 2, TSID_PATH_HYBRID = 3 } tsid_path_t;
 
 /* Sec. 5.3.  ASYM_STEP (default reading): D <- min(max(xi, -D), D) = min(D, xi): increases
  * of a coordinate are capped at eta*xi, decreases are free.  ASYM_GRAD: the same formula
@@ -228,6 +239,12 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
 /* Which path the handle runs (tsid_path_t, never AUTO) and how many kernels one
  * tsid_grad_step launches. */
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
+
+/* What the hybrid path stored (debug / bench surface): the number of 128 x 128 tiles kept densely, the
+ * smallest number of entries such a tile holds, and how many entries stayed on the gather-reduce passes.
+ * On a handle of another path all three are 0 (tail = nnz).  Any out pointer may be NULL. */
+tsid_status_t tsid_get_hybrid_info(const tsid_template_t *t, int64_t *h_tiles, int32_t *h_min_tile_entries,
+                                   int64_t *h_tail_entries);
 
 /* Template sampling (Sec. 5.1, "Sampling the TSID Template Submatrix"): the step before the
  * factorization.  Chooses d = ceil(alpha n) of the n columns uniformly at random without replacement

@@ -22,7 +22,7 @@ TSID_ERR_TOO_LARGE = 9
 (TSID_ERR_INVALID_ARG, TSID_ERR_INDEX_RANGE, TSID_ERR_DUPLICATE, TSID_ERR_UNSORTED, TSID_ERR_OOM,
  TSID_ERR_CUDA, TSID_ERR_UNSUPPORTED, TSID_ERR_NONFINITE) = range(1, 9)
 TSID_F32, TSID_BF16_SHADOW = 0, 1
-TSID_PATH_AUTO, TSID_PATH_SPARSE, TSID_PATH_DENSE_TC = 0, 1, 2
+TSID_PATH_AUTO, TSID_PATH_SPARSE, TSID_PATH_DENSE_TC, TSID_PATH_HYBRID = 0, 1, 2, 3
 TSID_CLIP_NONE, TSID_CLIP_ASYM_STEP, TSID_CLIP_ASYM_GRAD, TSID_CLIP_ASYM_ENTRY = 0, 1, 2, 3
 TSID_NORM_NONE, TSID_NORM_COUNT = 0, 1
 TSID_VALIDATE, TSID_INPUT_ROW_SORTED, TSID_VALUES_U8 = 1, 2, 4
@@ -33,7 +33,7 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
-           "tsid_set_norm_counts", "tsid_apply_sliced"]
+           "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info"]
 
 
 class TsidConfig(C.Structure):
@@ -87,6 +87,7 @@ def lib():
         L.tsid_residuals.argtypes = [vp, vp, vp, vp]
         L.tsid_get_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.tsid_last_error.argtypes = [vp]
+        L.tsid_get_hybrid_info.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
         L.tsid_workspace_bytes_host.argtypes = [C.POINTER(TsidConfig), C.POINTER(C.c_size_t)]
         L.tsid_fit_host.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, vp, C.c_int32, C.POINTER(C.c_double)]
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
@@ -257,6 +258,12 @@ class Template:
         p, l = C.c_int32(0), C.c_int32(0)
         lib().tsid_get_info(self.h, C.byref(p), C.byref(l))
         return p.value, l.value
+
+    def tsid_get_hybrid_info(self):
+        """(stored tiles, smallest entry count of a stored tile, entries left to the gather-reduce passes)."""
+        a, b, c = C.c_int64(0), C.c_int32(0), C.c_int64(0)
+        lib().tsid_get_hybrid_info(self.h, C.byref(a), C.byref(b), C.byref(c))
+        return a.value, b.value, c.value
 
     def tsid_set_profiling(self, enable):
         st = lib().tsid_set_profiling(self.h, int(enable))

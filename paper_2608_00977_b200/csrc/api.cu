@@ -22,12 +22,13 @@ tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
   if (c->m < 1 || c->n < 1 || c->nnz < 0) { snprintf(err, 256, "m, n must be >= 1 and nnz >= 0"); return TSID_ERR_INVALID_ARG; }
   if (c->nnz > 2147483647LL) { snprintf(err, 256, "nnz exceeds 2^31-1"); return TSID_ERR_UNSUPPORTED; }
   if (c->precision != TSID_F32 && c->precision != TSID_BF16_SHADOW) { snprintf(err, 256, "bad precision"); return TSID_ERR_INVALID_ARG; }
-  if (c->path < TSID_PATH_AUTO || c->path > TSID_PATH_DENSE_TC) { snprintf(err, 256, "bad path"); return TSID_ERR_INVALID_ARG; }
+  if (c->path < TSID_PATH_AUTO || c->path > TSID_PATH_HYBRID) { snprintf(err, 256, "bad path"); return TSID_ERR_INVALID_ARG; }
   if (c->clip < TSID_CLIP_NONE || c->clip > TSID_CLIP_ASYM_ENTRY) { snprintf(err, 256, "bad clip mode"); return TSID_ERR_INVALID_ARG; }
   if (c->norm_p < 0 || c->norm_p > 1 || c->norm_q < 0 || c->norm_q > 1) { snprintf(err, 256, "bad norm mode"); return TSID_ERR_INVALID_ARG; }
   const int mult = c->precision == TSID_BF16_SHADOW ? 8 : 4;
   if (c->k < 1 || c->k > 256 || c->k % mult) { snprintf(err, 256, "k must be in [1,256] and a multiple of %d", mult); return TSID_ERR_UNSUPPORTED; }
-  if (c->clip == TSID_CLIP_ASYM_ENTRY && (c->path == TSID_PATH_DENSE_TC || (c->precision == TSID_F32 && c->k > 128))) {
+  if (c->clip == TSID_CLIP_ASYM_ENTRY &&
+      (c->path == TSID_PATH_DENSE_TC || c->path == TSID_PATH_HYBRID || (c->precision == TSID_F32 && c->k > 128))) {
     snprintf(err, 256, "entry-wise clipping runs on the sparse path only (fp32 factors: k <= 128)");
     return TSID_ERR_UNSUPPORTED;
   }
@@ -35,12 +36,17 @@ tsid_status_t check_cfg(const tsid_config_t *c, char *err) {
   return TSID_OK;
 }
 
+// Below this many entries AUTO does not try the hybrid path: its extra launches per step cost more than
+// the tiles save.
+constexpr int64_t kHybridAutoMinEntries = 4000000;
+
 // AUTO takes the dense tensor-core variant when the template qualifies for it and at least 5 % of
 // its cells are observed; the answer depends on cfg alone, so the workspace size is predictable.
 int resolve_path(const tsid_config_t &c) {
   if (c.path != TSID_PATH_AUTO) return c.path;
   if (dense_qualifies(c) && c.clip != TSID_CLIP_ASYM_ENTRY && (double)c.nnz >= 0.05 * (double)c.m * (double)c.n)
     return TSID_PATH_DENSE_TC;
+  if (hybrid_qualifies(c) && c.nnz >= kHybridAutoMinEntries) return TSID_PATH_HYBRID;
   return TSID_PATH_SPARSE;
 }
 
@@ -80,11 +86,13 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
   t->red_cap = (int32_t)(2 + 2 * 256 + t->rowside.cap_seg);
   t->red = cv.take<double>(t->red_cap);
   if (t->path == TSID_PATH_DENSE_TC) dense_carve(t, c, cv);
-  // transient buffers of the layout pass
-  ls.kA = cv.take<uint32_t>(nz); ls.kB = cv.take<uint32_t>(nz);
-  ls.vA = cv.take<uint32_t>(nz); ls.vB = cv.take<uint32_t>(nz);
-  ls.wA = cv.take<uint32_t>(nz); ls.wB = cv.take<uint32_t>(nz);
-  ls.xA = cv.take<uint32_t>(nz); ls.xB = cv.take<uint32_t>(nz);
+  if (t->path == TSID_PATH_HYBRID) hybrid_carve(t, c, cv);
+  // buffers of the layout pass (one spare slot for the scans' totals); the hybrid path keeps its tail
+  // layout in four of them afterwards
+  ls.kA = cv.take<uint32_t>(nz + 64); ls.kB = cv.take<uint32_t>(nz + 64);
+  ls.vA = cv.take<uint32_t>(nz + 64); ls.vB = cv.take<uint32_t>(nz + 64);
+  ls.wA = cv.take<uint32_t>(nz + 64); ls.wB = cv.take<uint32_t>(nz + 64);
+  ls.xA = cv.take<uint32_t>(nz + 64); ls.xB = cv.take<uint32_t>(nz + 64);
   ls.hist = cv.take<uint32_t>(256 * (size_t)kSortBlocksMax);
   const size_t mx = (m > n ? m : n) + 2;
   ls.scanA = cv.take<uint32_t>(mx); ls.scanB = cv.take<uint32_t>(mx); ls.scanC = cv.take<uint32_t>(mx);
@@ -92,6 +100,7 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
 }
 
 cudaError_t grad_any(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ) {
+  if (t->path == TSID_PATH_HYBRID) return hybrid_grad(t, d_P, d_Q, GP, GQ);
   return t->path == TSID_PATH_DENSE_TC ? dense_grad(t, GP, GQ) : sparse_grad(t, d_P, d_Q, GP, GQ);
 }
 
@@ -168,6 +177,11 @@ tsid_status_t tsid_workspace_bytes(const tsid_config_t *cfg, size_t *h_bytes_out
     snprintf(g_create_err, 256, "dense path needs bf16 shadows, k in {64, 128}, m and n multiples of 128");
     return TSID_ERR_UNSUPPORTED;
   }
+  if (tmp.path == TSID_PATH_HYBRID && !hybrid_qualifies(*cfg)) {
+    snprintf(g_create_err, 256, "hybrid path needs bf16 shadows, k in {64, 128}, no entry-wise clip or byte values, "
+                                "and at least max(m, n, ceil(m/128) * ceil(n/128)) entries");
+    return TSID_ERR_UNSUPPORTED;
+  }
   Carver cv(nullptr);
   LayoutScratch ls;
   carve_all(&tmp, *cfg, cv, ls);
@@ -199,6 +213,10 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
     t->dense = dense_new();
     if (!t->dense) { delete t; return fail(nullptr, TSID_ERR_OOM, "host allocation failed"); }
   }
+  if (path == TSID_PATH_HYBRID) {
+    t->hybrid = hybrid_new();
+    if (!t->hybrid) { delete t; return fail(nullptr, TSID_ERR_OOM, "host allocation failed"); }
+  }
   Carver cv(cfg->workspace);
   LayoutScratch ls;
   carve_all(t, *cfg, cv, ls);
@@ -223,6 +241,12 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
     e = dense_build(t, &bad);
     if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
     if (bad) { tsid_destroy(t); return fail(nullptr, TSID_ERR_UNSUPPORTED, "a value is outside the fp16 range of the dense path"); }
+  }
+  if (path == TSID_PATH_HYBRID) {
+    int32_t fallback = 0;
+    e = hybrid_build(t, ls, &fallback);
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+    if (fallback) t->path = TSID_PATH_SPARSE;   // no tile worth storing (or duplicates, or a value beyond fp16)
   }
   snprintf(t->err, 256, "ok");
   *out = t;
@@ -385,7 +409,7 @@ static void prof_release(tsid_template *t) {
 }
 
 tsid_status_t tsid_destroy(tsid_template_t *t) {
-  if (t) { prof_release(t); fit_graph_release(t); dense_delete(t->dense); }
+  if (t) { prof_release(t); fit_graph_release(t); dense_delete(t->dense); hybrid_delete(t->hybrid); }
   delete t;
   return TSID_OK;
 }
@@ -536,7 +560,22 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step) {
   if (!t) return TSID_ERR_INVALID_ARG;
   if (h_path) *h_path = t->path;
-  if (h_launches_per_step) *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? dense_launches_per_step(t) : sparse_launches_per_step(t);
+  if (h_launches_per_step) {
+    if (t->path == TSID_PATH_HYBRID) *h_launches_per_step = 1 + hybrid_launches_per_step(t) + 1;   // + shadow refresh, update
+    else *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? dense_launches_per_step(t) : sparse_launches_per_step(t);
+  }
+  return TSID_OK;
+}
+
+tsid_status_t tsid_get_hybrid_info(const tsid_template_t *t, int64_t *h_tiles, int32_t *h_min_tile_entries,
+                                   int64_t *h_tail_entries) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  int64_t tiles = 0, tail = t->cfg.nnz;
+  int32_t mine = 0;
+  if (t->path == TSID_PATH_HYBRID) hybrid_info(t, &tiles, &mine, &tail);
+  if (h_tiles) *h_tiles = tiles;
+  if (h_min_tile_entries) *h_min_tile_entries = mine;
+  if (h_tail_entries) *h_tail_entries = tail;
   return TSID_OK;
 }
 

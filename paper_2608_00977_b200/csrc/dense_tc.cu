@@ -87,7 +87,8 @@ template <int K>
 __global__ void __launch_bounds__(576, 1)
 dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ CUtensorMap tmY,
                   const __grid_constant__ CUtensorMap tmR, int rows_x, int rows_y, int nsplit,
-                  float *__restrict__ G, float *__restrict__ Gpart, int32_t *__restrict__ flags) {
+                  float *__restrict__ G, float *__restrict__ Gpart, int32_t *__restrict__ flags,
+                  const DenseChunk *__restrict__ chunks, const int32_t *__restrict__ ylist) {
   using L = Smem<K>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;   // tiles need 1024-byte alignment
@@ -97,12 +98,25 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ib = blockIdx.x / nsplit, sp = blockIdx.x % nsplit;
-  const int row0 = ib * BLK;
-  const int NJ = rows_y / BLK;
-  const int jb0 = (int)((long long)NJ * sp / nsplit), jb1 = (int)((long long)NJ * (sp + 1) / nsplit);
-  const int NW = jb1 - jb0;                // work items of this CTA
-  float *Gout = sp == 0 ? G : Gpart + (size_t)(sp - 1) * rows_x * K;
+  // Whole-matrix form: CTA (ib, sp) walks the column blocks [jb0, jb0 + NW) of a dense R.  Tile-list form
+  // (chunks != nullptr): the CTA walks the NW stored tiles [t0, t0 + NW) of row block ib; tile t holds the
+  // cells of (ib, ylist[t]) as one 128 x 128 block of the tile array behind tmR, and the CTA's result is a
+  // partial gradient block of its own (the caller adds the blocks of a row block in chunk order).
+  int row0, jb0, NW, t0 = 0;
+  float *Gout;           // where row `row0 + r` of this CTA's result goes: Gout + (grow0 + r) * K
+  int grow0;
+  if (chunks) {
+    const DenseChunk ck = chunks[blockIdx.x];
+    row0 = ck.ib * BLK; jb0 = 0; NW = ck.nt; t0 = ck.t0;
+    Gout = Gpart + (size_t)ck.slot * BLK * K; grow0 = 0;
+  } else {
+    const int ib = blockIdx.x / nsplit, sp = blockIdx.x % nsplit;
+    row0 = ib * BLK;
+    const int NJ = rows_y / BLK;
+    jb0 = (int)((long long)NJ * sp / nsplit);
+    NW = (int)((long long)NJ * (sp + 1) / nsplit) - jb0;
+    Gout = sp == 0 ? G : Gpart + (size_t)(sp - 1) * rows_x * K; grow0 = row0;
+  }
 
   if (threadIdx.x == 0) {
     mbar_init(bar(L::B_XFULL), 8);
@@ -128,8 +142,10 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
   if (warp == 0) {
     // ---- TMA producer ---------------------------------------------------------------------------
     if (lane == 0) {
+      int jb_next = (ylist && NW > 0) ? __ldg(ylist + t0) : jb0;
       for (int w = 0; w < NW && ok; ++w) {
-        const int jb = jb0 + w, ys = w % L::NSY, rs = w % L::NSR;
+        const int jb = jb_next, ys = w % L::NSY, rs = w % L::NSR;
+        if (w + 1 < NW) jb_next = ylist ? __ldg(ylist + t0 + w + 1) : jb + 1;
         if (w >= L::NSY) ok = mbar_wait(bar(L::B_YEMPTY + ys), ((w / L::NSY) - 1) & 1);
         if (!ok) break;
         mbar_expect_tx(bar(L::B_YFULL + ys), L::Y_BYTES);
@@ -138,8 +154,10 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
         if (w >= L::NSR) ok = mbar_wait(bar(L::B_REMPTY + rs), ((w / L::NSR) - 1) & 1);
         if (!ok) break;
         mbar_expect_tx(bar(L::B_RFULL + rs), L::R_BYTES);
-        for (int c = 0; c < 2; ++c)
-          tma_load_2d(sm0 + L::OFF_R + rs * L::R_BYTES + c * L::XB, &tmR, bar(L::B_RFULL + rs), jb * BLK + c * 64, row0);
+        for (int c = 0; c < 2; ++c) {
+          if (chunks) tma_load_2d(sm0 + L::OFF_R + rs * L::R_BYTES + c * L::XB, &tmR, bar(L::B_RFULL + rs), c * 64, (t0 + w) * BLK);
+          else tma_load_2d(sm0 + L::OFF_R + rs * L::R_BYTES + c * L::XB, &tmR, bar(L::B_RFULL + rs), jb * BLK + c * 64, row0);
+        }
       }
     }
     __syncwarp();
@@ -253,7 +271,7 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
     if (ok && writer) ok = __all_sync(0xffffffffu, mbar_wait(bar(L::B_GFULL), 0));
     if (ok && writer) {
       tc_fence_after();
-      float *grow = Gout + (size_t)(row0 + row) * K + h * (K / 2);
+      float *grow = Gout + (size_t)(grow0 + row) * K + h * (K / 2);
 #pragma unroll
       for (int c = 0; c < K / 64; ++c) {
         uint32_t gv[32];
@@ -328,7 +346,7 @@ cudaError_t launch_dense_pass(cudaStream_t st, const __nv_bfloat16 *X, const CUt
   auto kern = dense_pass_kernel<K>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<K>::TOTAL));
   const int nrb = rows_x / BLK, nsplit = dense_split(rows_x, rows_y);
-  kern<<<nrb * nsplit, 576, Smem<K>::TOTAL, st>>>(X, tmY, tmR, rows_x, rows_y, nsplit, G, Gpart, flags);
+  kern<<<nrb * nsplit, 576, Smem<K>::TOTAL, st>>>(X, tmY, tmR, rows_x, rows_y, nsplit, G, Gpart, flags, nullptr, nullptr);
   if (nsplit > 1) {
     const size_t n4 = (size_t)rows_x * K / 4;
     add_partials_kernel<<<148 * 4, 256, 0, st>>>(reinterpret_cast<float4 *>(G), reinterpret_cast<const float4 *>(Gpart),
@@ -379,6 +397,29 @@ cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag) {
 int dense_launches_per_step(const tsid_template *t) {
   const tsid_config_t &c = t->cfg;
   return 4 + (dense_split(c.m, c.n) > 1) + (dense_split(c.n, c.m) > 1);
+}
+
+cudaError_t dense_make_map(void *map, bool half_not_bf16, void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  return make_map(reinterpret_cast<CUtensorMap *>(map),
+                  half_not_bf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, rows, cols, box_rows);
+}
+
+cudaError_t dense_tiles_pass(cudaStream_t st, int k, const __nv_bfloat16 *X, const void *map_y, const void *map_r,
+                             const DenseChunk *chunks, int nchunks, const int32_t *ylist, float *partial, int32_t *flags) {
+  if (nchunks <= 0) return cudaSuccess;
+  const CUtensorMap &tmY = *reinterpret_cast<const CUtensorMap *>(map_y);
+  const CUtensorMap &tmR = *reinterpret_cast<const CUtensorMap *>(map_r);
+  if (k == 128) {
+    auto kern = dense_pass_kernel<128>;
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::TOTAL));
+    kern<<<nchunks, 576, Smem<128>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist);
+  } else {
+    auto kern = dense_pass_kernel<64>;
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::TOTAL));
+    kern<<<nchunks, 576, Smem<64>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist);
+  }
+  return cudaGetLastError();
 }
 
 // G_P and G_Q from the current bf16 shadows (which must be up to date).

@@ -401,7 +401,7 @@ __global__ void seg_count_kernel(const int64_t *__restrict__ ptr, int32_t nrows,
     nslot[i] = s > 1 ? s : 0u;
     nsplit[i] = s > 1 ? 1u : 0u;
     float sc = (norm_count && cnt > 1) ? (float)cnt : 1.0f;
-    scale[i] = 2.0f / sc;
+    if (scale) scale[i] = 2.0f / sc;   // null: segments of a side whose normalisation is kept elsewhere
   }
 }
 

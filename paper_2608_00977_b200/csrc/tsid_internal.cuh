@@ -50,12 +50,19 @@ struct Side {
   int32_t cap_seg = 0, cap_split = 0, cap_slot = 0;
 };
 
-struct DenseState;  // dense_tc.cu
+struct DenseState;   // dense_tc.cu
+struct HybridState;  // hybrid.cu
+
+// One CTA's share of a tile-list pass of the tensor-core kernel: the stored tiles [t0, t0 + nt) of row
+// block ib; the CTA's partial gradient block goes to slot `slot` of the partial buffer.
+struct __align__(16) DenseChunk {
+  int32_t ib, t0, nt, slot;
+};
 
 // Optional per-kernel timing: CUDA events recorded on the template's stream right around the
 // row pass, the column pass and the update kernel of each step (up to kProfSteps steps).
 constexpr int kProfSteps = 256;
-enum { EV_ROW0 = 0, EV_ROW1, EV_COL0, EV_COL1, EV_UPD0, EV_UPD1, EV_PER_STEP };
+enum { EV_ROW0 = 0, EV_ROW1, EV_COL0, EV_COL1, EV_UPD0, EV_UPD1, EV_DNS0, EV_DNS1, EV_PER_STEP };
 struct Prof {
   bool on = false;
   int nsteps = 0;
@@ -79,6 +86,7 @@ struct tsid_template {
   int32_t red_cap;
   int32_t *flags;     // device flags: [0] range, [1] unsorted, [2] duplicate, [3] non-finite
   tsid::DenseState *dense;
+  tsid::HybridState *hybrid;
   tsid::Prof prof;
   // tsid_fit replays its epochs from an executable graph: fit_steps steps on the factor arrays
   // fit_P / fit_Q, captured on fit_cap (no work ever runs there) and kept until arrays or count change
@@ -177,6 +185,23 @@ void dense_carve(tsid_template *t, const tsid_config_t &c, Carver &cv);
 cudaError_t dense_build(tsid_template *t, int32_t *h_range_flag);
 int dense_launches_per_step(const tsid_template *t);
 cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ);
+// tensor map (128 bytes at `map`) of a 16-bit matrix [rows][cols], box = box_rows x 64 columns, 128-byte swizzle
+cudaError_t dense_make_map(void *map, bool half_not_bf16, void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// tile-list pass: partial[chunk.slot] = sum over the chunk's tiles of (M .* (R_tile - X_blk Y_blk^T)) Y_blk
+cudaError_t dense_tiles_pass(cudaStream_t st, int k, const __nv_bfloat16 *X, const void *map_y, const void *map_r,
+                             const DenseChunk *chunks, int nchunks, const int32_t *ylist, float *partial, int32_t *flags);
+
+// hybrid path (hybrid.cu): the populated 128 x 128 tiles of the degree-ordered template on the tensor cores,
+// every other entry through the gather-reduce passes
+bool hybrid_qualifies(const tsid_config_t &c);
+HybridState *hybrid_new();
+void hybrid_delete(HybridState *h);
+void hybrid_carve(tsid_template *t, const tsid_config_t &c, Carver &cv);
+// builds the tiles and the tail layout; *h_status: 0 ok, 1 no tile worth it (or duplicates / fp16 range): run sparse
+cudaError_t hybrid_build(tsid_template *t, LayoutScratch &s, int32_t *h_status);
+cudaError_t hybrid_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ);
+int hybrid_launches_per_step(const tsid_template *t);
+void hybrid_info(const tsid_template *t, int64_t *tiles, int32_t *min_entries, int64_t *tail);
 
 inline int bits_for(uint32_t maxval) {  // number of bits needed to represent values <= maxval
   int b = 0;
