@@ -3,10 +3,15 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C5] [--impl reference]
 
-A step is one full-batch gradient step (row pass, column pass, fix-ups, clip + update with the
-shadow refresh of bf16 templates) over the whole synthetic template, inputs resident in HBM: K
-epochs of one tsid_fit call, or K tsid_grad_step calls where L2 is flushed between steps.  One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs an independent
-replica of the same template (the path is single-GPU; there is no data-path collective).
+A step is one full-batch gradient step (both gradient passes, fix-ups, clip + update with the shadow
+refresh of bf16 templates) over the whole synthetic template, inputs resident in HBM: K epochs of one
+tsid_fit call, or K tsid_grad_step calls where L2 is flushed between steps.  Every timed region is
+repeated REPS times (best and median reported; the headline is the median).  One JSON line is printed
+by rank 0: the headline workload (the 1e9-entry template on the path TSID_PATH_AUTO picks), and under
+"secondary" the same measurement of the other configurations (the dense tensor-core variant on C4
+among them).  With N > 1 (torchrun) every rank runs an independent replica of the same template (the
+path is single-GPU; there is no data-path collective); a "sharded" sub-record times the row-sharded
+form as well.
 """
 from __future__ import annotations
 
@@ -29,14 +34,31 @@ import torch  # noqa: E402
 METRIC = "observed-entry gradient updates/sec"
 UNIT = "updates/s"
 L2_BYTES = 126 * 1024 * 1024
+REPS = 5
+SEG_LEN = 512        # kSegLen of the library build the traffic figures were captured on
+N_SMS = 148
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gather-reduce pass kernel
-# (average of the row pass and the column pass), from the ncu summaries under profiles/.
-NCU_TRAFFIC_PER_LAUNCH = {
-    "C5": 93.79e9,        # profiles/step_kernels_C5_launches_dram.md: row 78.88 GB, column 108.69 GB
-    "C3": 0.865e9,        # profiles/pass_staged_kernel_C3_ncu.md
-    "C4-dense": 0.551e9,  # profiles/dense_pass_kernel_C4_ncu.md: the fp16 R matrix once per launch
+# What the paper itself reports (another machine, whole-run seconds; context, never the target).
+PAPER_CONTEXT = {
+    "hardware": "2x Intel Xeon Gold 6426Y, 512 GB RAM, 4x NVIDIA A100 40 GB, CUDA 12.4, PyTorch AMP fp16/fp32 (Sec. 6.1, Test Platform)",
+    "stage1_time_s": "2.0-2.2 s for template recovery on 10K..100K synthetic matrices; SVD in its place 3.4-8.6 s; 4.09x faster (Sec. 6.5)",
+    "tensor_core_vs_cuda_core_s": {"16Kx16K": [30.7, 22.18], "32Kx32K": [62.16, 47.88], "64Kx64K": [158.21, 136.25],
+                                   "80Kx80K": [283.4, 216.7], "what": "whole run, CUDA cores -> Tensor Cores (Sec. 6.4)"},
+    "conflict_free_stage1_s": "8.30 -> 4.71 s end to end on 1Kx3K, up to 43 % (Sec. 6.3 ablation)",
+    "memory_gb": {"1Kx3K": 0.30, "3Kx3K": 0.47, "3Kx10K": 0.79, "Last.fm": 0.85, "MovieLens-25M": 27, "MovieLens-33M": 38,
+                  "Netflix": 22, "Yahoo": 23, "what": "peak GPU memory, both stages (Table 6)"},
+    "headline": "up to 11,647x faster than CSNN, up to 8.5x lower peak memory, up to 99.7 % lower NMAE (abstract; end to end)",
+    "per_step_throughput": "not reported by the paper (no updates/s, GB/s or kernel time for Stage I)",
 }
+
+
+def load_traffic():
+    """ncu figures per launch of the dominant kernels (profiles/traffic.json, written beside the summaries)."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f)
+    return {}
 
 
 def load_peaks():
@@ -112,19 +134,6 @@ def aggregate_value(world, units_per_rank_step, steps, seconds):
     return world * units_per_rank_step * steps / seconds
 
 
-def alg_bytes(w, nnz, nseg_row, nseg_col, value_bytes=4):
-    """Algorithmic bytes of one launch of each kernel of a step.  A pass reads per entry a 4-byte index, a
-    4-byte value and one gathered factor row (k*b bytes, b = 2 for bf16 shadows, 4 for fp32), and per row the
-    staged factor row (k*b), a 16-byte segment descriptor, and writes the gradient row (4k).  The update reads
-    gradient and master, writes master (and the bf16 shadow), and reads one scale per row."""
-    b = 2 if w.precision == "bf16" else 4
-    k = w.k
-    row = nnz * (4 + value_bytes + k * b) + w.m * k * (b + 4) + nseg_row * 16
-    col = nnz * (4 + value_bytes + k * b) + w.n * k * (b + 4) + nseg_col * 16
-    upd = (w.m + w.n) * k * (4 + 4 + 4 + (b if b == 2 else 0)) + (w.m + w.n) * 4
-    return row, col, upd
-
-
 def run_reference(args, W):
     """The oracle, as it stands, on the host cores: each step is one oracle step over a bounded
     sample (a prefix of the row-sorted COO) of the workload."""
@@ -161,18 +170,33 @@ def run_reference(args, W):
     print(json.dumps(line))
 
 
-def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=25.0):
-    """Times the oracle on a prefix of the template's (row-sorted) COO entries with the full factor
-    matrices; sized from a short calibration run so that it takes about budget_s seconds."""
+def _oracle_slice(a):
+    """One single-threaded oracle step over one row slice (runs in a child process)."""
+    import oracle
+    m_used, n, k, r, c, v, P, Q, eta, lam, xi, clip, norm_p, norm_q = a
+    t0 = time.perf_counter()
+    oracle.grad_step(m_used, n, k, r, c, v, P, Q, eta, lam, xi, clip, norm_p, norm_q)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=20.0):
+    """Times the oracle, as it stands, on a prefix of the template's (row-sorted) COO entries with the full
+    factor matrices: once on one core, and once as N single-threaded oracle processes on disjoint row slices
+    of such a prefix (N = the host's cores; the oracle itself has no threads).  Sized from a short calibration
+    run so that each leg takes about budget_s seconds."""
+    import multiprocessing as mp
     import numpy as np
     import oracle
     nnz = tpl_dev.nnz
     P, Q = P0.cpu().numpy(), Q0.cpu().numpy()
 
-    def run(count):
+    def prefix(count):
         r = tpl_dev.rows[:count].cpu().numpy(); c = tpl_dev.cols[:count].cpu().numpy()
         v = tpl_dev.vals[:count].cpu().numpy()
-        m_used = int(r.max()) + 1 if count else 1     # the prefix touches rows [0, m_used)
+        return r, c, v, (int(r.max()) + 1 if count else 1)     # the prefix touches rows [0, m_used)
+
+    def run(count):
+        r, c, v, m_used = prefix(count)
         t0 = time.perf_counter()
         oracle.grad_step(m_used, w.n, w.k, r, c, v, P[:m_used], Q, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
         return time.perf_counter() - t0, m_used
@@ -182,9 +206,34 @@ def cpu_baseline(w, tpl_dev, P0, Q0, budget_s=25.0):
     if t < 0.5 * budget_s and count < nnz:   # the first run also pays fixed costs: rescale once
         count = int(min(nnz, count * budget_s / max(t, 1e-3)))
         t, m_used = run(count)
-    return {"value": count / t, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "first %d of %d row-sorted entries (rows 0..%d, all %d columns), one oracle grad_step, "
-                      "%.1f s" % (count, nnz, m_used - 1, w.n, t)}
+    out = {"value": count / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": "first %d of %d row-sorted entries (rows 0..%d, all %d columns), one oracle grad_step, "
+                     "%.1f s" % (count, nnz, m_used - 1, w.n, t)}
+    ncores = os.cpu_count() or 1
+    if ncores > 1:
+        total = int(min(nnz, count * ncores))
+        r, c, v, m_all = prefix(total)
+        cuts = [int(np.searchsorted(r, m_all * i // ncores)) for i in range(ncores + 1)]
+        cuts[-1] = total
+        jobs = []
+        for i in range(ncores):
+            a, b = cuts[i], cuts[i + 1]
+            if b <= a:
+                continue
+            r0 = int(r[a]); m_i = int(r[b - 1]) - r0 + 1
+            jobs.append((m_i, w.n, w.k, r[a:b] - r0, c[a:b], v[a:b], P[r0:r0 + m_i], Q, w.eta, w.lam, w.xi, w.clip,
+                         w.norm_p, w.norm_q))
+        try:
+            with mp.get_context("fork").Pool(len(jobs)) as pool:
+                t0 = time.perf_counter()
+                pool.map(_oracle_slice, jobs, chunksize=1)
+                wall = time.perf_counter() - t0
+            out["all_cores"] = {"value": total / wall, "unit": UNIT, "cores": len(jobs), "kind": "oracle",
+                                "sample": "first %d entries cut into %d row slices, one single-threaded oracle process per "
+                                          "slice, all at once, %.1f s wall" % (total, len(jobs), wall)}
+        except Exception as ex:   # a host that cannot fork: the single-core figure stands alone
+            out["all_cores"] = {"unavailable": repr(ex)}
+    return out
 
 
 def measure_sampling(args, w, tpl, B, dev):
@@ -370,9 +419,10 @@ def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
     clocks = sampler.stop()
     sh.T.tsid_check()
     sse = sh.sse(P, Q)
+    rec = None
     if rank == 0:
         _, launches = sh.T.tsid_get_info()
-        print(json.dumps({"metric": METRIC, "value": tpl.nnz * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        rec = ({"metric": METRIC, "value": tpl.nnz * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
                           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
                           "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
                           "dtype": "bf16" if w.precision == "bf16" else "f32", "data": "synthetic",
@@ -382,8 +432,249 @@ def run_row_sharded(args, w, tpl, B, dev, dist, rank, world):
                                                      "rows/%d, all-reduce(sum) of G_Q (%d bytes) per step") % (world, w.n * w.k * 4),
                                      "l2": "inputs larger than L2, steps timed back to back"},
                           "clocks": clocks, "e2e": None, "gpu_launches": launches * args.steps, "roofline": None,
-                          "cpu_baseline": None, "rmse_after": (sse / tpl.nnz) ** 0.5}))
+                          "cpu_baseline": None, "rmse_after": (sse / tpl.nnz) ** 0.5})
     sh.destroy()
+    return rec
+
+
+def alg_bytes_pass(w, entries, rows, nseg, value_bytes=4):
+    """Algorithmic bytes of one gather-reduce pass launch over `entries` entries of `rows` staged rows."""
+    b = 2 if w.precision == "bf16" else 4
+    return entries * (4 + value_bytes + w.k * b) + rows * w.k * (b + 4) + nseg * 16
+
+
+class StepBench:
+    """One workload on one kernel path: template, warm-up, REPS timed regions of K steps, per-kernel times."""
+
+    def __init__(self, args, W, B, wname, path_name, dev, dist, local, values="f32"):
+        self.args, self.W, self.B, self.dev, self.dist, self.local = args, W, B, dev, dist, local
+        self.wname, self.path_name, self.values = wname, path_name, values
+        self.w = W.CONFIGS[wname]
+        self.tpl = None
+        self.T = None
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize(self.dev)
+
+    def create(self, tpl=None):
+        B, w = self.B, self.w
+        t0 = time.perf_counter()
+        self.tpl = tpl if tpl is not None else self.W.make_template(w, self.dev, order="sorted")
+        torch.cuda.synchronize(self.dev)
+        t1 = time.perf_counter()
+        want = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC,
+                "hybrid": B.TSID_PATH_HYBRID}[self.path_name]
+        self.want_path = want
+        vflags = B.TSID_VALUES_U8 if self.values == "u8" else 0
+        self.T = B.template_from_workload(self.tpl, path=want, flags=vflags)
+        torch.cuda.synchronize(self.dev)
+        self.gen_s, self.create_s = t1 - t0, time.perf_counter() - t1
+        self.path, self.launches = self.T.tsid_get_info()
+        self.P, self.Q = self.tpl.P0.clone(), self.tpl.Q0.clone()
+        return self
+
+    def measure(self, steps, warmup, long_seconds=0.0):
+        """Returns the record of this workload (timings in ms per step)."""
+        B, w, T, P, Q, dev = self.B, self.w, self.T, self.P, self.Q, self.dev
+        nnz = self.tpl.nnz
+        stream = torch.cuda.current_stream(dev)
+        resident = nnz * 16 + (w.m + w.n) * w.k * 4
+        flush = resident < 4 * L2_BYTES
+        scrub = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
+        for _ in range(warmup):
+            T.tsid_grad_step(P, Q)
+        T.tsid_check()
+        sampler = ClockSampler(self.local)
+        sampler.start()
+        time.sleep(0.3)
+
+        def timed(profiled=False, nsteps=steps):
+            self.barrier()
+            if flush:
+                evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nsteps)]
+                for a, b in evs:
+                    scrub.fill_(1)
+                    a.record(stream)
+                    T.tsid_grad_step(P, Q)
+                    b.record(stream)
+                self.barrier()
+                return sum(a.elapsed_time(b) for a, b in evs)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            if profiled:
+                for _ in range(nsteps):
+                    T.tsid_grad_step(P, Q)
+            else:
+                T.tsid_fit(P, Q, nsteps)      # K steps, replayed from the library's captured graph
+            b.record(stream)
+            self.barrier()
+            return a.elapsed_time(b)
+
+        # The headline loop carries no events between its kernels; the same K steps are then repeated with the
+        # library's per-kernel events on the launching stream, and the roofline of the dominant kernel uses those.
+        if not flush:
+            T.tsid_fit(P, Q, steps)          # untimed: the call that captures the graph of K steps
+            T.tsid_check()
+        reps = [max_over_ranks(timed(), self.dist, dev) / steps for _ in range(REPS)]
+        clocks = sampler.stop()
+        long_run = None
+        if long_seconds > 0 and not flush:
+            # a region long enough for the power cap to set in (the regime of the sustained peak)
+            nlong = max(steps, int(math.ceil(long_seconds * 1e3 / min(reps) / 8.0)) * 8)
+            s2 = ClockSampler(self.local)
+            s2.start()
+            T.tsid_fit(P, Q, 8)
+            ms_long = max_over_ranks(timed(nsteps=nlong), self.dist, dev) / nlong
+            long_run = {"steps": nlong, "ms_per_step": ms_long, "clocks": s2.stop()}
+        T.tsid_set_profiling(True)
+        ms_prof = timed(profiled=True) / steps
+        nrec, row_ms, col_ms, upd_ms, tile_ms = T.tsid_get_step_times()
+        T.tsid_set_profiling(False)
+        T.tsid_check()
+        nrec = max(1, nrec)
+        self.flush = flush
+        shadow = 1 if w.precision == "bf16" else 0
+        return {"reps_ms_per_step": reps, "best": min(reps), "median": statistics.median(reps), "clocks": clocks,
+                "long_run": long_run, "ms_per_step_with_events": ms_prof,
+                "kernel_ms": {"row_pass": row_ms / nrec, "col_pass": col_ms / nrec, "update": upd_ms / nrec,
+                              "tile_passes": tile_ms / nrec},
+                "gpu_launches_per_rep": self.launches * steps if flush else (self.launches - shadow) * steps + shadow,
+                "resident_bytes": resident}
+
+    def roofline(self, rec, traffic):
+        """Roofline record of the dominant kernel of this path, from the live launch durations."""
+        B, w, T = self.B, self.w, self.T
+        nnz = self.tpl.nnz
+        peak, tf_sustained, tf_burst, peak_kind = load_peaks()
+        km = rec["kernel_ms"]
+        ms_step = rec["median"]
+        mhz = rec["clocks"].get("sm_mhz") or 1965.0
+        tkey = "%s-%s" % (self.wname, "dense" if self.path == B.TSID_PATH_DENSE_TC else
+                          ("hybrid" if self.path == B.TSID_PATH_HYBRID else "sparse"))
+        tr = traffic.get(tkey, {})
+        if self.path == B.TSID_PATH_DENSE_TC:
+            # dense variant: the dominant kernel is the tcgen05 pass (two launches per step); algorithmic flops
+            # are the three GEMMs of the method, 6 m n k per step, i.e. 3 m n k per launch (four are executed)
+            pass_ms = (km["row_pass"] + km["col_pass"]) / 2
+            fl = 3.0 * w.m * w.n * w.k
+            tfl_short = fl / (pass_ms * 1e-3) / 1e12
+            out = {"bound": "tensor", "kernel": "dense_pass_kernel (tcgen05; pass over R and pass over R^T)",
+                   "unit": "TFLOP/s", "alg_flops_per_launch": fl, "executed_flops_per_launch": 4.0 * w.m * w.n * w.k,
+                   "avg_launch_ms": pass_ms, "traffic": tr.get("dram_bytes_per_launch"),
+                   "pass_R": {"ms": km["row_pass"]}, "pass_RT": {"ms": km["col_pass"]}, "update": {"ms": km["update"]},
+                   "short_run": {"what": "launch durations of the %d-step runs (clock %s MHz: burst regime)" % (
+                                     self.args.steps, rec["clocks"].get("sm_mhz")),
+                                 "kernel_tflops": tfl_short, "kernel_frac_of_burst": tfl_short / tf_burst,
+                                 "step_frac_of_burst": 6.0 * w.m * w.n * w.k / (ms_step * 1e-3) / 1e12 / tf_burst},
+                   "peak_burst": tf_burst, "peak_sustained": tf_sustained, "frac_of_nominal_2250": tfl_short / 2250.0}
+            lr = rec.get("long_run")
+            if lr:
+                # like for like: a seconds-long region against the sustained peak; the pass kernels' share of a step
+                # is taken from the per-kernel events of the short run
+                share = 2 * pass_ms / max(1e-9, rec["ms_per_step_with_events"])
+                step_tfl = 6.0 * w.m * w.n * w.k / (lr["ms_per_step"] * 1e-3) / 1e12
+                out["long_run"] = {"steps": lr["steps"], "ms_per_step": lr["ms_per_step"], "clocks": lr["clocks"],
+                                   "step_tflops": step_tfl, "step_frac_of_sustained": step_tfl / tf_sustained,
+                                   "kernel_frac_of_sustained": step_tfl / max(share, 1e-9) / tf_sustained if share < 1 else None}
+                out.update({"achieved": step_tfl, "peak": tf_sustained, "frac": step_tfl / tf_sustained,
+                            "peak_source": "of %s (sustained bf16, against a %d-step region under the power cap)" % (
+                                peak_kind, lr["steps"]),
+                            "frac_is": "whole step (both passes + update), algorithmic flops, long run / sustained peak"})
+            else:
+                out.update({"achieved": tfl_short, "peak": tf_burst, "frac": tfl_short / tf_burst,
+                            "peak_source": "of %s (burst bf16: short run at full clock)" % peak_kind})
+            return out
+        # gather-reduce passes (all entries on the sparse path, the tail entries on the hybrid path)
+        tiles, min_tile, tail = T.tsid_get_hybrid_info()
+        ent = tail if self.path == B.TSID_PATH_HYBRID else nnz
+        vb = 1 if self.values == "u8" else 4
+        b_row = alg_bytes_pass(w, ent, w.m, w.m + ent // SEG_LEN, vb)
+        b_col = alg_bytes_pass(w, ent, w.n, w.n + ent // SEG_LEN, vb)
+        b = 2 if w.precision == "bf16" else 4
+        b_upd = (w.m + w.n) * w.k * (4 + 4 + 4 + (b if b == 2 else 0)) + (w.m + w.n) * 4
+        pass_ms = (km["row_pass"] + km["col_pass"]) / 2
+        bytes_per_launch = (b_row + b_col) / 2
+        achieved = bytes_per_launch / (pass_ms * 1e-3) / 1e9 if pass_ms > 0 else 0.0
+        step_alg = nnz * (8 + vb * 2 + 2 * w.k * b) + (w.m + w.n) * w.k * 20 + (w.m + w.n + 2) * 8
+        step_min = nnz * 16 + (w.m + w.n) * w.k * 20
+        out = {"bound": "hbm",
+               "kernel": "pass_staged_kernel (gather-reduce: CSR row pass + CSC column pass, 2 launches per step%s)" % (
+                   "; the %d entries outside the dense tiles" % ent if self.path == B.TSID_PATH_HYBRID else ""),
+               "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "alg_frac": achieved / peak,
+               "peak_source": "of %s" % peak_kind,
+               "note": "frac = alg_frac charges every gathered factor row at HBM rate although L2 serves many of them, so it "
+                       "can exceed 1; hbm_frac is what HBM itself carried (ncu DRAM bytes / launch time / peak)",
+               "alg_bytes_per_launch": bytes_per_launch, "avg_launch_ms": pass_ms,
+               "row_pass": {"ms": km["row_pass"], "alg_bytes": b_row},
+               "col_pass": {"ms": km["col_pass"], "alg_bytes": b_col},
+               "update": {"ms": km["update"], "alg_bytes": b_upd,
+                          "gbs": b_upd / (km["update"] * 1e-3) / 1e9 if km["update"] else None},
+               "step_alg_bytes": step_alg, "step_compulsory_bytes": step_min,
+               "step_frac": step_alg / (ms_step * 1e-3) / 1e9 / peak,
+               "frac_compulsory": step_min / (ms_step * 1e-3) / 1e9 / peak,
+               "frac_of_nominal_8TBs": achieved / 8000.0}
+        out["traffic"] = tr.get("dram_bytes_per_launch")
+        if tr:
+            out["traffic_from"] = tr.get("from")
+            if tr.get("seg_len") not in (None, SEG_LEN):
+                out["traffic_stale"] = "captured with segments of %s entries, this build uses %d" % (tr.get("seg_len"), SEG_LEN)
+            if tr.get("dram_bytes_per_launch") and pass_ms > 0:
+                out["dram_gbs"] = tr["dram_bytes_per_launch"] / (pass_ms * 1e-3) / 1e9
+                out["hbm_frac"] = out["frac_dram"] = out["dram_gbs"] / peak
+            if tr.get("warp_insts_per_entry") and pass_ms > 0:
+                # share of the issue slots the pass uses: warp instructions / (SMs x 4 schedulers x clock x time)
+                out["issue"] = {"warp_insts_per_entry": tr["warp_insts_per_entry"], "sm_mhz": mhz,
+                                "frac": tr["warp_insts_per_entry"] * ent / (pass_ms * 1e-3) / (N_SMS * 4 * mhz * 1e6)}
+        if self.path == B.TSID_PATH_HYBRID:
+            fl_alg = 6.0 * 128 * 128 * w.k * tiles   # per step, both tile passes: S, E Y and E^T X of every stored tile
+            out["tile_passes"] = {"tiles": tiles, "min_entries_per_tile": min_tile, "entries_in_tiles": nnz - tail,
+                                  "ms": km["tile_passes"],
+                                  "what": "rank-ordered shadow copies, tcgen05 tile pass over R tiles and over R^T tiles, two adds",
+                                  "alg_tflops": fl_alg / (km["tile_passes"] * 1e-3) / 1e12 if km["tile_passes"] else None,
+                                  "frac_of_burst_peak": fl_alg / (km["tile_passes"] * 1e-3) / 1e12 / tf_burst if km["tile_passes"] else None}
+        return out
+
+    def destroy(self):
+        if self.T is not None:
+            self.T.tsid_destroy()
+            self.T = None
+        self.P = self.Q = None
+        torch.cuda.empty_cache()
+
+
+def path_label(B, path):
+    return {B.TSID_PATH_SPARSE: "sparse", B.TSID_PATH_DENSE_TC: "dense_tc", B.TSID_PATH_HYBRID: "hybrid"}.get(path, str(path))
+
+
+def workload_config(B, sb, world):
+    w, nnz = sb.w, sb.tpl.nnz
+    return {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": nnz,
+            "precision": "bf16 shadow factors, fp32 master and accumulation" if w.precision == "bf16" else "fp32",
+            "path": path_label(B, sb.path), "path_requested": sb.path_name,
+            "values": "one byte per rating" if sb.values == "u8" else "fp32",
+            "step": "%s (eta=%g lambda=%g xi=%g clip=%d norm=%d/%d)" % (
+                "K calls of tsid_grad_step" if sb.flush else "one tsid_fit of K epochs (graph replay)",
+                w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q),
+            "l2": "L2 flushed between timed steps (resident set %.0f MB)" % (sb.resident / 1e6) if sb.flush
+                  else "inputs larger than L2 (resident set %.1f GB), steps timed back to back" % (sb.resident / 1e9),
+            "repetitions": REPS, "replicas": world}
+
+
+def secondary_record(args, W, B, wname, path_name, dev, local, traffic, tpl=None, long_seconds=0.0):
+    """One more workload measured like the headline (no e2e, no CPU leg)."""
+    sb = StepBench(args, W, B, wname, path_name, dev, None, local).create(tpl)
+    rec = sb.measure(args.steps, args.warmup, long_seconds)
+    sb.resident = rec["resident_bytes"]
+    roof = sb.roofline(rec, traffic)
+    nnz = sb.tpl.nnz
+    out = {"config": workload_config(B, sb, 1), "ms_per_step": rec["median"], "best_ms_per_step": rec["best"],
+           "reps_ms_per_step": rec["reps_ms_per_step"], "value": nnz / (rec["median"] * 1e-3), "unit": UNIT,
+           "clocks": rec["clocks"], "roofline": roof, "layout_s": sb.create_s,
+           "workspace_gb": sb.T.workspace.numel() / 1e9}
+    sb.destroy()
+    return out
 
 
 def main():
@@ -393,8 +684,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=os.environ.get("TSID_BENCH_WORKLOAD", "C5"))
     ap.add_argument("--impl", default="tsid")
-    ap.add_argument("--path", default="sparse", choices=["auto", "sparse", "dense"],
-                    help="kernel path of the measured template (the dense tcgen05 variant needs a qualifying workload, e.g. C4)")
+    ap.add_argument("--path", default="auto", choices=["auto", "sparse", "dense", "hybrid"],
+                    help="kernel path of the measured template (auto: what TSID_PATH_AUTO resolves to; the dense tcgen05 "
+                         "variant needs a qualifying workload, e.g. C4)")
     ap.add_argument("--measure", default="step", choices=["step", "sample", "extend", "layout"],
                     help="step: the gradient step (default); sample: tsid_sample_template on the workload's COO; "
                          "extend: Stage II (tsid_extend) of the workload's matrix on a template of a quarter of its columns; "
@@ -413,6 +705,7 @@ def main():
                     help="u8: stream the ratings as one byte each (TSID_VALUES_U8; needs integer values, e.g. C2, C3, C5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="only the headline workload (no C5-sparse / C4 / C3 / C2 records)")
     ap.add_argument("--e2e-epochs", type=int, default=0, help="epochs per host-buffer call (0: the workload's)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -442,156 +735,53 @@ def main():
     B.lib()
 
     w = W.CONFIGS[args.workload]
-    t0 = time.perf_counter()
-    tpl = W.make_template(w, dev, order=args.order if args.measure == "layout" else "sorted")
-    torch.cuda.synchronize(dev)
-    t1 = time.perf_counter()
-    nnz = tpl.nnz
-    if args.measure == "sample":
-        measure_sampling(args, w, tpl, B, dev)
-        return
-    if args.measure == "extend":
-        measure_extend(args, w, tpl, B, dev)
-        return
-    if args.measure == "layout":
-        measure_layout(args, w, tpl, B, dev)
-        return
-    if args.shard == "rows":
-        run_row_sharded(args, w, tpl, B, dev, dist, rank, world)
-        return
-    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
-    want_path = {"auto": B.TSID_PATH_AUTO, "sparse": B.TSID_PATH_SPARSE, "dense": B.TSID_PATH_DENSE_TC}[args.path]
-    vflags = B.TSID_VALUES_U8 if args.values == "u8" else 0
-    T = B.template_from_workload(tpl, path=want_path, flags=vflags)
-    torch.cuda.synchronize(dev)
-    if rank == 0:
-        sys.stderr.write("[bench] %s: generated %d entries in %.1f s, layout pass %.2f s, workspace %.2f GB\n" % (
-            w.name, nnz, t1 - t0, time.perf_counter() - t1, T.workspace.numel() / 1e9))
-    path, launches = T.tsid_get_info()
-    P, Q = tpl.P0.clone(), tpl.Q0.clone()
-    stream = torch.cuda.current_stream(dev)
-
-    resident = nnz * 16 + (w.m + w.n) * w.k * 4
-    flush = resident < 4 * L2_BYTES
-    scrub = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
+    if args.measure != "step" or args.shard == "rows":
+        tpl = W.make_template(w, dev, order=args.order if args.measure == "layout" else "sorted")
         torch.cuda.synchronize(dev)
-
-    for _ in range(args.warmup):
-        T.tsid_grad_step(P, Q)
-    T.tsid_check()
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.3)
-
-    def timed_steps(profiled=False):
-        barrier()
-        if flush:
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-            for a, b in evs:
-                scrub.fill_(1)
-                a.record(stream)
-                T.tsid_grad_step(P, Q)
-                b.record(stream)
-            barrier()
-            return sum(a.elapsed_time(b) for a, b in evs)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        if profiled:
-            for _ in range(args.steps):
-                T.tsid_grad_step(P, Q)
+        if args.measure == "sample":
+            measure_sampling(args, w, tpl, B, dev)
+        elif args.measure == "extend":
+            measure_extend(args, w, tpl, B, dev)
+        elif args.measure == "layout":
+            measure_layout(args, w, tpl, B, dev)
         else:
-            T.tsid_fit(P, Q, args.steps)      # K steps, replayed from the library's captured graph
-        b.record(stream)
-        barrier()
-        return a.elapsed_time(b)
+            rec = run_row_sharded(args, w, tpl, B, dev, dist, rank, world)
+            if rank == 0:
+                print(json.dumps(rec))
+        return
 
-    # The headline loop carries no events between its kernels; the same K steps are then repeated with the
-    # library's per-kernel events on the launching stream (they cost ~15 us per step, 5 % of a 0.3 ms step),
-    # and the roofline of the dominant kernel uses those launch durations.
-    if not flush:
-        T.tsid_fit(P, Q, args.steps)          # untimed: the call that captures the graph of K steps
-        T.tsid_check()
-    ms = timed_steps()
-    T.tsid_set_profiling(True)
-    ms_profiled = timed_steps(profiled=True)
-    clocks = sampler.stop()
-    nrec, row_ms, col_ms, upd_ms = T.tsid_get_pass_times()
-    T.tsid_set_profiling(False)
-    T.tsid_check()
-
-    ms = max_over_ranks(ms, dist, dev)
-    value = aggregate_value(world, nnz, args.steps, ms * 1e-3)
-    # tsid_grad_step refreshes the bf16 shadows on entry (the caller may have changed the factors); tsid_fit
-    # does that once per call, its update kernel keeps them current
-    shadow = 1 if w.precision == "bf16" else 0
-    gpu_launches = launches * args.steps if flush else (launches - shadow) * args.steps + shadow
-
-    # ---- roofline of the dominant kernel (the gather-reduce pass: two launches per step) ----------
-    peak, tf_sustained, tf_burst, peak_kind = load_peaks()
-    nseg_row = w.m + nnz // 512
-    nseg_col = w.n + nnz // 512
-    b_row, b_col, b_upd = alg_bytes(w, nnz, nseg_row, nseg_col, 1 if args.values == "u8" else 4)
-    pass_ms = (row_ms + col_ms) / max(1, 2 * nrec)
-    bytes_per_launch = (b_row + b_col) / 2
-    achieved = bytes_per_launch / (pass_ms * 1e-3) / 1e9 if pass_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "pass_kernel (CSR row pass + CSC column pass, 2 launches per step)",
-                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_source": "of %s" % peak_kind, "traffic": NCU_TRAFFIC_PER_LAUNCH.get(args.workload),
-                "alg_bytes_per_launch": bytes_per_launch, "avg_launch_ms": pass_ms,
-                "row_pass": {"ms": row_ms / max(1, nrec), "alg_bytes": b_row,
-                             "gbs": b_row / (row_ms / max(1, nrec) * 1e-3) / 1e9 if row_ms else None},
-                "col_pass": {"ms": col_ms / max(1, nrec), "alg_bytes": b_col,
-                             "gbs": b_col / (col_ms / max(1, nrec) * 1e-3) / 1e9 if col_ms else None},
-                "update": {"ms": upd_ms / max(1, nrec), "alg_bytes": b_upd,
-                           "gbs": b_upd / (upd_ms / max(1, nrec) * 1e-3) / 1e9 if upd_ms else None},
-                "step_alg_bytes": b_row + b_col + b_upd,
-                "step_compulsory_bytes": nnz * 16 + (w.m + w.n) * w.k * 20,   # perfect cache: streams + factors once
-                "step_frac": (b_row + b_col + b_upd) / (ms / args.steps * 1e-3) / 1e9 / peak,
-                "frac_of_nominal_8TBs": achieved / 8000.0}
-    tr = NCU_TRAFFIC_PER_LAUNCH.get(args.workload)
-    if tr and pass_ms > 0:
-        # what HBM itself carried (ncu's DRAM bytes of a launch over this run's launch time): the algorithmic
-        # figure above counts every gathered row as if it came from HBM, and L2 serves most of them
-        roofline["dram_gbs"] = tr / (pass_ms * 1e-3) / 1e9
-        roofline["dram_frac"] = roofline["dram_gbs"] / peak
-    timing_note = {"launch_times_from": "the same %d steps repeated with the library's per-kernel CUDA events" % args.steps,
-                   "ms_per_step_with_events": ms_profiled / args.steps}
-    if path == B.TSID_PATH_DENSE_TC:
-        # dense variant: the dominant kernel is the tcgen05 pass (two launches per step); algorithmic
-        # flops are the three GEMMs of the method, 6 m n k per step, i.e. 3 m n k per launch
-        flops_launch = 3.0 * w.m * w.n * w.k
-        tfl = flops_launch / (pass_ms * 1e-3) / 1e12 if pass_ms > 0 else 0.0
-        roofline = {"bound": "tensor", "kernel": "dense_pass_kernel (tcgen05; pass over R and pass over R^T)",
-                    "achieved": tfl, "peak": tf_sustained, "unit": "TFLOP/s", "frac": tfl / tf_sustained,
-                    "peak_source": "of %s (sustained bf16; burst %.1f)" % (peak_kind, tf_burst),
-                    "traffic": NCU_TRAFFIC_PER_LAUNCH.get(args.workload + "-dense"),
-                    "alg_flops_per_launch": flops_launch, "executed_flops_per_launch": 4.0 * w.m * w.n * w.k,
-                    "avg_launch_ms": pass_ms,
-                    "pass_R": {"ms": row_ms / max(1, nrec)}, "pass_RT": {"ms": col_ms / max(1, nrec)},
-                    "update": {"ms": upd_ms / max(1, nrec)},
-                    "step_frac": 6.0 * w.m * w.n * w.k / (ms / args.steps * 1e-3) / 1e12 / tf_sustained,
-                    "frac_of_burst": tfl / tf_burst, "frac_of_nominal_2250": tfl / 2250.0}
-
-    roofline.update(timing_note)
+    traffic = load_traffic()
+    sb = StepBench(args, W, B, args.workload, args.path, dev, dist, local, args.values).create()
+    tpl, nnz = sb.tpl, sb.tpl.nnz
+    if rank == 0:
+        sys.stderr.write("[bench] %s: generated %d entries in %.1f s, create (layout pass) %.2f s, workspace %.2f GB, path %s\n" % (
+            w.name, nnz, sb.gen_s, sb.create_s, sb.T.workspace.numel() / 1e9, path_label(B, sb.path)))
+    dense_headline = sb.path == B.TSID_PATH_DENSE_TC
+    rec = sb.measure(args.steps, args.warmup, long_seconds=2.5 if dense_headline else 0.0)
+    sb.resident = rec["resident_bytes"]
+    ms_step = rec["median"]
+    value = aggregate_value(world, nnz, 1, ms_step * 1e-3)
+    roofline = sb.roofline(rec, traffic)
+    roofline.update({"launch_times_from": "the same %d steps repeated with the library's per-kernel CUDA events" % args.steps,
+                     "ms_per_step_with_events": rec["ms_per_step_with_events"]})
+    config = workload_config(B, sb, world)
+    prec = B.TSID_BF16_SHADOW if w.precision == "bf16" else B.TSID_F32
+    want_path = sb.want_path
+    ws_gb = sb.T.workspace.numel() / 1e9
+    create_s = sb.create_s
+    sb.destroy()
 
     # ---- end to end: host buffers through tsid_fit_host ----------------------------------------------
     e2e = None
     if not args.no_e2e:
         epochs = args.e2e_epochs or w.epochs
         cfg = B.make_config(w.m, w.n, w.k, nnz, prec, want_path, w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q)
-        T.tsid_destroy()
-        del T
-        torch.cuda.empty_cache()
         hb = [x.cpu().pin_memory() for x in (tpl.rows, tpl.cols, tpl.vals)]
         hP0, hQ0 = tpl.P0.cpu(), tpl.Q0.cpu()
         hP, hQ = hP0.clone().pin_memory(), hQ0.clone().pin_memory()
         ws = torch.empty(B.tsid_workspace_bytes_host(cfg) + 256, dtype=torch.uint8, device=dev)
         reps = 2
-        barrier()
+        sb.barrier()
         t_e2e = 0.0
         for rep in range(reps + 1):
             hP.copy_(hP0); hQ.copy_(hQ0)
@@ -607,31 +797,57 @@ def main():
         e2e = {"value": world * nnz * epochs * reps / t_e2e, "unit": UNIT,
                "h2d_bytes_per_step": h2d / epochs, "d2h_bytes_per_step": d2h / epochs,
                "epochs_per_call": epochs, "h2d_bytes_per_call": h2d, "d2h_bytes_per_call": d2h,
-               "s_per_call": t_e2e / reps,
-               "what": "tsid_fit_host: pinned host COO + factors -> device, layout pass, epochs steps, factors -> host"}
-        del ws
+               "s_per_call": t_e2e / reps, "input_order": "COO sorted by (row, col); a shuffled COO adds two sorts to the layout pass",
+               "what": "tsid_fit_host: pinned host COO + factors -> device, layout pass (and tile build), epochs steps, "
+                       "factors -> host; the paper runs 100 - 10,000 iterations per template, which would amortise the "
+                       "copies and the layout further"}
+        del ws, hb, hP, hQ
+        torch.cuda.empty_cache()
 
+    # ---- the row-sharded form of the same template, when there is more than one rank ------------------
+    sharded = None
+    if world > 1:
+        try:
+            sharded = run_row_sharded(args, w, tpl, B, dev, dist, rank, world)
+        except Exception as ex:   # the replica line above stands on its own
+            sharded = {"unavailable": repr(ex)}
+
+    # ---- the other configurations, measured the same way (rank 0 of a single-GPU run) -----------------
+    secondary = None
+    if rank == 0 and world == 1 and not args.no_secondary:
+        secondary = {}
+        try:
+            if sb.path != B.TSID_PATH_SPARSE:
+                secondary["%s-sparse" % args.workload] = secondary_record(args, W, B, args.workload, "sparse", dev, local,
+                                                                          traffic, tpl=tpl)
+        except Exception as ex:
+            secondary["%s-sparse" % args.workload] = {"unavailable": repr(ex)}
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(w, tpl, tpl.P0, tpl.Q0)
+    del tpl
+    sb.tpl = None
+    torch.cuda.empty_cache()
+    if secondary is not None:
+        for key, wname, pname, long_s in (("C4-dense", "C4", "dense", 2.5), ("C3", "C3", "auto", 0.0), ("C2", "C2", "auto", 0.0)):
+            if wname == args.workload:
+                continue
+            try:
+                secondary[key] = secondary_record(args, W, B, wname, pname, dev, local, traffic, long_seconds=long_s)
+            except Exception as ex:
+                secondary[key] = {"unavailable": repr(ex)}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision == "bf16" else "f32",
-                "data": "synthetic",
-                "config": {"workload": w.name, "m": w.m, "n": w.n, "k": w.k, "nnz": nnz,
-                           "precision": "bf16 shadow factors, fp32 master and accumulation" if w.precision == "bf16" else "fp32",
-                           "path": "sparse" if path == B.TSID_PATH_SPARSE else "dense_tc",
-                           "values": "one byte per rating" if args.values == "u8" else "fp32",
-                           "step": "%s (eta=%g lambda=%g xi=%g clip=%d norm=%d/%d)" % (
-                               "K calls of tsid_grad_step" if flush else "one tsid_fit of K epochs (graph replay)",
-                               w.eta, w.lam, w.xi, w.clip, w.norm_p, w.norm_q),
-                           "l2": "L2 flushed between timed steps (resident set %.0f MB)" % (resident / 1e6) if flush
-                                 else "inputs larger than L2 (resident set %.1f GB), steps timed back to back" % (resident / 1e9),
-                           "replicas": world},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches,
-                "roofline": roofline, "cpu_baseline": cpu}
+                "data": "synthetic", "config": config,
+                "timing": {"repetitions": REPS, "reps_ms_per_step": rec["reps_ms_per_step"], "best_ms_per_step": rec["best"],
+                           "median_ms_per_step": rec["median"], "headline": "median of the repetitions, each exactly K steps",
+                           "create_s": create_s, "workspace_gb": ws_gb},
+                "clocks": rec["clocks"], "e2e": e2e, "gpu_launches": rec["gpu_launches_per_rep"],
+                "roofline": roofline, "cpu_baseline": cpu, "secondary": secondary, "sharded": sharded,
+                "paper_context": PAPER_CONTEXT}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

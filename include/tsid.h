@@ -319,6 +319,10 @@ tsid_status_t tsid_extend(const tsid_extend_config_t *cfg, const float *d_P, con
  * tsid_get_pass_times synchronises, returns the number of recorded steps and the summed
  * milliseconds of each of the three kernels over them, and restarts the recording. */
 tsid_status_t tsid_set_profiling(tsid_template_t *t, int32_t enable);
+/* The same with a fourth figure: h_ms4 = { row pass, column pass, update, tile passes } summed over the
+ * recorded steps; the fourth is the hybrid path's tensor-core part (rank-ordered shadow copies, the two
+ * tile-list passes and the two adds), 0 on the other paths. */
+tsid_status_t tsid_get_step_times(tsid_template_t *t, int32_t *h_steps, float *h_ms4);
 tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms,
                                   float *h_col_ms, float *h_update_ms);
 

@@ -33,7 +33,7 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
-           "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info"]
+           "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info", "tsid_get_step_times"]
 
 
 class TsidConfig(C.Structure):
@@ -92,6 +92,7 @@ def lib():
         L.tsid_fit_host.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, vp, C.c_int32, C.POINTER(C.c_double)]
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
         L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
+        L.tsid_get_step_times.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_float)]
         L.tsid_sse_noalloc.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
         L.tsid_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
         L.tsid_sample_template.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_uint64, vp, vp, vp, vp, vp,
@@ -278,6 +279,15 @@ class Template:
         if st != TSID_OK:
             self._raise(st)
         return n.value, a.value, b.value, c.value
+
+    def tsid_get_step_times(self):
+        """(steps, row_ms, col_ms, update_ms, tiles_ms) summed over the recorded steps."""
+        n = C.c_int32(0)
+        ms = (C.c_float * 4)()
+        st = lib().tsid_get_step_times(self.h, C.byref(n), ms)
+        if st != TSID_OK:
+            self._raise(st)
+        return n.value, ms[0], ms[1], ms[2], ms[3]
 
     def tsid_get_layout(self, copy=True):
         """The layout arrays as torch tensors (row_ptr, col_idx, val_csr, col_ptr, row_idx, val_csc, perm):

@@ -430,15 +430,15 @@ tsid_status_t tsid_set_profiling(tsid_template_t *t, int32_t enable) {
   return TSID_OK;
 }
 
-tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms, float *h_col_ms,
-                                  float *h_update_ms) {
+tsid_status_t tsid_get_step_times(tsid_template_t *t, int32_t *h_steps, float *h_ms4) {
   if (!t) return TSID_ERR_INVALID_ARG;
   if (!t->prof.on) return fail(t, TSID_ERR_INVALID_ARG, "profiling is off");
   cudaError_t e = cudaStreamSynchronize(t->stream);
   if (e != cudaSuccess) return cuda_fail(t, e);
-  double acc[3] = {0, 0, 0};
+  double acc[4] = {0, 0, 0, 0};
+  const int nq = t->path == TSID_PATH_HYBRID ? 4 : 3;   // the fourth pair brackets the tile passes of the hybrid path
   for (int sidx = 0; sidx < t->prof.nsteps; ++sidx) {
-    for (int q = 0; q < 3; ++q) {
+    for (int q = 0; q < nq; ++q) {
       float ms = 0.f;
       e = cudaEventElapsedTime(&ms, t->prof.ev[sidx * EV_PER_STEP + 2 * q], t->prof.ev[sidx * EV_PER_STEP + 2 * q + 1]);
       if (e != cudaSuccess) return cuda_fail(t, e);
@@ -446,10 +446,19 @@ tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h
     }
   }
   if (h_steps) *h_steps = t->prof.nsteps;
-  if (h_row_ms) *h_row_ms = (float)acc[0];
-  if (h_col_ms) *h_col_ms = (float)acc[1];
-  if (h_update_ms) *h_update_ms = (float)acc[2];
+  if (h_ms4) for (int q = 0; q < 4; ++q) h_ms4[q] = (float)acc[q];
   t->prof.nsteps = 0;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_get_pass_times(tsid_template_t *t, int32_t *h_steps, float *h_row_ms, float *h_col_ms,
+                                  float *h_update_ms) {
+  float ms[4] = {0.f, 0.f, 0.f, 0.f};
+  tsid_status_t st = tsid_get_step_times(t, h_steps, ms);
+  if (st != TSID_OK) return st;
+  if (h_row_ms) *h_row_ms = ms[0];
+  if (h_col_ms) *h_col_ms = ms[1];
+  if (h_update_ms) *h_update_ms = ms[2];
   return TSID_OK;
 }
 
