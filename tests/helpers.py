@@ -18,6 +18,20 @@ def relerr(a, ref):
     return float(np.max(np.abs(a - ref)) / den) if ref.size else 0.0
 
 
+def rowwise_relerr(a, ref, counts):
+    """Per-row check: max_i |a_i - ref_i|_inf / max(|ref_i|_inf, floor_i).  The whole-matrix metric above lets the
+    most populated rows set the scale; here every row is held to its own size.  A row whose terms cancel has no
+    relative accuracy of its own, so the denominator never goes below the size a sum of count_i random-sign
+    terms has: floor_i = sqrt(max(count_i, 1)) * t, t = the median over rows of |ref_i|_inf / sqrt(count_i)."""
+    a = np.asarray(a, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    if ref.size == 0:
+        return 0.0
+    c = np.sqrt(np.maximum(np.asarray(counts, dtype=np.float64), 1.0))
+    mag = np.max(np.abs(ref), axis=1)
+    t = np.median((mag / c)[mag > 0]) if np.any(mag > 0) else 1.0
+    return float(np.max(np.max(np.abs(a - ref), axis=1) / np.maximum(mag, c * t)))
+
+
 def np_coo(tpl):
     return (tpl.rows.cpu().numpy(), tpl.cols.cpu().numpy(), tpl.vals.cpu().numpy())
 

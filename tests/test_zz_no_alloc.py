@@ -4,7 +4,8 @@ Such callers (a hook inside a process whose framework has reserved the whole GPU
 plug-in that only receives pointers and a stream) cannot build a workspace for tsid_loss.  The variant
 keeps its reduction scratch in a fixed array inside the library.  Here it is called through the C ABI
 twice in a row (the second call finds the first call's leftovers in the scratch) and compared with what
-tsid_loss returns for the same template, at the tolerance the loss tests use (1e-5 relative).
+tsid_loss returns for the same template and with the CPU oracle's loss, at the tolerance the loss tests
+use (1e-5 relative).
 
 This file sorts last on purpose, so that a run that stops at the first failure has already run the rest.
 """
@@ -14,7 +15,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import small_workload
+import oracle
+from helpers import np_coo, small_workload
 from paper_2608_00977_b200 import binding as B
 from paper_2608_00977_b200 import workloads as W
 
@@ -47,6 +49,14 @@ def test_noalloc_sse_matches_tsid_loss_on_two_calls_in_a_row():
     T.tsid_destroy()
     got2 = _sse_noalloc(big, tpls[0], P2, Q2)
     for g, r in zip(got + [got2], refs + [ref2]):
+        assert r > 0 and abs(g - r) / r <= 1e-5, (g, r)
+    # and against the CPU oracle's loss (double sums over the COO triples), at the same tolerance
+    orc = []
+    for w, tpl, scale in ((big, tpls[0], 1.0), (small, tpls[1], 1.0), (big, tpls[0], 0.5)):
+        r, c, v = np_coo(tpl)
+        orc.append(oracle.loss(w.m, w.n, w.k, r, c, v, tpl.P0.cpu().numpy() * np.float32(scale),
+                               tpl.Q0.cpu().numpy() * np.float32(scale), 0.0)[0])
+    for g, r in zip(got + [got2], orc):
         assert r > 0 and abs(g - r) / r <= 1e-5, (g, r)
     # deterministic: the same call again gives the same bits
     assert _sse_noalloc(big, tpls[0], P2, Q2) == got2
