@@ -128,22 +128,29 @@ typedef struct {
   size_t workspace_bytes; /* its size                                                     */
 } tsid_config_t;
 
-/* Bytes of device workspace a template with cfg's m, n, k, nnz, precision and path needs.
- * Reads only those fields.  Host-only, no CUDA call. */
+/* Bytes of device workspace a template needs (no counterpart in the paper: the library allocates nothing, the
+ * caller brings the memory).  The size depends on m, n, k, nnz, precision, path (AUTO resolves from these and
+ * clip), and flags (TSID_VALUES_U8 adds two byte streams); the whole cfg is validated as by
+ * tsid_template_create, so fill every field the way the create call will see it (stream, workspace and
+ * workspace_bytes are not read).  Host-only, no CUDA call.  Errors: INVALID_ARG, UNSUPPORTED. */
 tsid_status_t tsid_workspace_bytes(const tsid_config_t *cfg, size_t *h_bytes_out);
 
-/* Layout pass + handle creation.  d_rows, d_cols (int32[nnz]) and d_vals (fp32[nnz]) are
+/* Layout pass + handle creation: takes the problem as Def. 1 / Sec. 1 state it - R in R^{m x n} known on the
+ * index set Omega - with Omega given as COO triples (Sec. 6.1, "Data Model").  d_rows, d_cols (int32[nnz]) and d_vals (fp32[nnz]) are
  * the COO triples of Omega on the DEVICE, in any order; they are only read, and may be
  * freed when the call returns (it synchronises cfg.stream).  Builds in the workspace:
  * CSR sorted by (row, col), CSC sorted by (col, row), perm (CSC position -> CSR position),
  * the equal-length work segments of both passes, gradient / shadow / partial buffers.
- * Duplicates, when not rejected by TSID_VALIDATE, are each counted; ties keep input order.
+ * Duplicates, when not rejected by TSID_VALIDATE, are each counted; ties keep input order.  A dense cell
+ * holds one value, so TSID_PATH_DENSE_TC refuses a template with a duplicate (TSID_ERR_DUPLICATE, whatever
+ * the flags say) and TSID_PATH_HYBRID runs such a template on the sparse path.
  * On error *out is NULL. */
 tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_rows,
                                    const int32_t *d_cols, const float *d_vals,
                                    tsid_template_t **out);
 
-/* One full-batch step, in place on d_P (m x k) and d_Q (n x k).  If d_gradP / d_gradQ are
+/* One full-batch step (Sec. 5.1 Eqs. (update-p), (update-q) summed over Omega, aggregated as in Eq. 9 with its
+ * 1/n normalisation; clip of Sec. 5.3), in place on d_P (m x k) and d_Q (n x k).  If d_gradP / d_gradQ are
  * non-null they receive the raw sums G_P = E Q (m x k) and G_Q = E^T P (n x k), fp32,
  * computed from the factors as they were BEFORE the update.  Asynchronous. */
 tsid_status_t tsid_grad_step(tsid_template_t *t, float *d_P, float *d_Q, float *d_gradP_or_null,
@@ -183,7 +190,8 @@ tsid_status_t tsid_apply_sliced(tsid_template_t *t, float *d_P, const float *d_G
 tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or_null,
                                    const int32_t *d_cnt_q_or_null);
 
-/* `epochs` steps in place.  loss_every > 0: after every loss_every-th step (and before the
+/* The iteration of Sec. 5.1, "Stage I Execution Example" (repeat the step until R* ~ P Q^T; here a fixed number
+ * of epochs): `epochs` steps in place.  loss_every > 0: after every loss_every-th step (and before the
  * first) the SSE is computed and stored in h_sse_history_or_null (host, capacity
  * 1 + epochs / loss_every doubles); this synchronises.  loss_every == 0: asynchronous.
  *   With loss_every == 0 and epochs >= 4 the steps are replayed from an executable CUDA graph (the
@@ -219,7 +227,7 @@ tsid_status_t tsid_fit_host(const tsid_config_t *cfg, const int32_t *h_rows, con
                             const float *h_vals, float *h_P, float *h_Q, int32_t epochs,
                             double *h_sse_or_null);
 
-/* Releases the host handle.  The workspace belongs to the caller.  NULL is accepted. */
+/* Releases the host handle (no counterpart in the paper).  The workspace belongs to the caller.  NULL is accepted. */
 tsid_status_t tsid_destroy(tsid_template_t *t);
 
 /* ---- debug / test surface ------------------------------------------------------------ */
@@ -245,6 +253,16 @@ tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *
  * On a handle of another path all three are 0 (tail = nnz).  Any out pointer may be NULL. */
 tsid_status_t tsid_get_hybrid_info(const tsid_template_t *t, int64_t *h_tiles, int32_t *h_min_tile_entries,
                                    int64_t *h_tail_entries);
+
+/* Test hook for the failure path of the tensor-core kernel (no counterpart in the paper).  Every wait of that
+ * kernel on one of its barriers is bounded by a cycle budget; when it runs out the CTA raises a flag, stops
+ * issuing work, frees its tensor memory and returns, and the next synchronising call reports TSID_ERR_CUDA
+ * ("a bounded device-side wait expired").  This call makes that happen on purpose, without faulting anything:
+ * from now on the kernels of this handle (TSID_PATH_DENSE_TC only, else TSID_ERR_UNSUPPORTED) use a budget of
+ * `wait_cycles` clock cycles and their load-issuing thread stops before work item `item` of each CTA, so the
+ * consumers of that item wait for loads that were never issued (nothing is outstanding).  wait_cycles = 0
+ * restores normal operation.  The gradients of a stalled step are meaningless. */
+tsid_status_t tsid_debug_stall_tile_pass(tsid_template_t *t, int64_t wait_cycles, int32_t item);
 
 /* Template sampling (Sec. 5.1, "Sampling the TSID Template Submatrix"): the step before the
  * factorization.  Chooses d = ceil(alpha n) of the n columns uniformly at random without replacement

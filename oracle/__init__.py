@@ -20,6 +20,8 @@ _LIB = os.path.join(_HERE, "libtsid_oracle.so")
 
 CLIP_NONE, CLIP_ASYM_STEP, CLIP_ASYM_GRAD, CLIP_ASYM_ENTRY = 0, 1, 2, 3
 NORM_NONE, NORM_COUNT = 0, 1
+# levels of the emulation switch (argument bf16_emulate; True means EMU_BF16)
+EMU_NONE, EMU_BF16, EMU_TENSOR = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -41,6 +43,8 @@ def _L():
         _lib = C.CDLL(build())
         _lib.orc_bf16_round.restype = C.c_float
         _lib.orc_bf16_round.argtypes = [C.c_float]
+        _lib.orc_fp16_round.restype = C.c_float
+        _lib.orc_fp16_round.argtypes = [C.c_float]
         _lib.orc_clip_nested.restype = C.c_double
         _lib.orc_clip_nested.argtypes = [C.c_double, C.c_double]
     return _lib
@@ -66,6 +70,10 @@ def _fac(X, nrow, k):
 
 def bf16_round(x: float) -> float:
     return float(_L().orc_bf16_round(C.c_float(x)))
+
+
+def fp16_round(x: float) -> float:
+    return float(_L().orc_fp16_round(C.c_float(x)))
 
 
 def clip_nested(g: float, xi: float) -> float:

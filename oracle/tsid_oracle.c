@@ -37,6 +37,13 @@
  *     row without entries does not move.  The "gradient sums" returned in this mode are the
  *     sums of the c_ij.
  *
+ * The emulation switch (argument bf16_emulate) has three levels: 0 reads the fp32 values; 1 rounds every factor
+ * value read to bfloat16 (what the gather-reduce passes of a bf16 template read); 2 is what the tensor-core
+ * variant forms (Sec. 5.1, half-precision multiplicands, fp32 accumulation): factors rounded to bfloat16, the
+ * observed value r rounded to binary16, and the residual e rounded to bfloat16 before it multiplies a factor
+ * row in the two gradient sums.  Level 2 acts on orc_residuals, orc_grad_sums and the aggregated modes of
+ * orc_grad_step; the loss and the entry-wise clip treat it as level 1.
+ *
  * Pins: every function below is pinned by tests marked "not gpu" (hand-worked
  * 3x2 and 8x6 examples stored as golden text, finite differences of the loss,
  * zero gradient at the true factors, the dense special case against numpy,
@@ -75,6 +82,26 @@ float orc_bf16_round(float x) {
   return y;
 }
 
+/* Round a float to the nearest IEEE-754 binary16 value (ties to even) and return it as float.  Values that
+ * round beyond the largest half (65504) become infinity; below 2^-14 the half grid is k * 2^-24. */
+float orc_fp16_round(float x) {
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  uint32_t a = u & 0x7fffffffu;
+  if (a >= 0x7f800000u) return x;                       /* inf / nan */
+  if (a < 0x38800000u) {                                /* |x| < 2^-14: subnormal halves */
+    double q = rint((double)x * 16777216.0);            /* nearest even multiple of 2^-24 (default rounding mode) */
+    return (float)(q / 16777216.0);
+  }
+  uint32_t lsb = (u >> 13) & 1u;
+  u += 0x0fffu + lsb;
+  u &= 0xffffe000u;
+  if ((u & 0x7fffffffu) >= 0x47800000u) u = (u & 0x80000000u) | 0x7f800000u;   /* 65520 and beyond: infinity */
+  float y;
+  memcpy(&y, &u, 4);
+  return y;
+}
+
 /* Sec. 5.3: the nested clip, written exactly as printed. */
 double orc_clip_nested(double g, double xi) {
   double a = (xi > -g) ? xi : -g;   /* max(xi, -g) */
@@ -98,7 +125,8 @@ void orc_residuals(int32_t m, int32_t n, int32_t k, int64_t nnz,
     double dot = 0.0;
     for (int32_t l = 0; l < k; ++l)
       dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
-    e_out[t] = (double)vals[t] - dot;
+    if (bf16_emulate == 2) e_out[t] = (double)orc_bf16_round((float)((double)orc_fp16_round(vals[t]) - dot));
+    else e_out[t] = (double)vals[t] - dot;
   }
 }
 
@@ -118,6 +146,7 @@ void orc_grad_sums(int32_t m, int32_t n, int32_t k, int64_t nnz,
     for (int32_t l = 0; l < k; ++l)
       dot += read_factor(P, i * k + l, bf16_emulate) * read_factor(Q, j * k + l, bf16_emulate);
     double e = (double)vals[t] - dot;
+    if (bf16_emulate == 2) e = (double)orc_bf16_round((float)((double)orc_fp16_round(vals[t]) - dot));
     for (int32_t l = 0; l < k; ++l) {
       GP[i * k + l] += e * read_factor(Q, j * k + l, bf16_emulate);
       GQ[j * k + l] += e * read_factor(P, i * k + l, bf16_emulate);

@@ -33,7 +33,8 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_last_error", "tsid_workspace_bytes_host", "tsid_fit_host", "tsid_set_profiling",
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
-           "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info", "tsid_get_step_times"]
+           "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info", "tsid_get_step_times",
+           "tsid_debug_stall_tile_pass"]
 
 
 class TsidConfig(C.Structure):
@@ -92,6 +93,7 @@ def lib():
         L.tsid_fit_host.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, vp, C.c_int32, C.POINTER(C.c_double)]
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
         L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
+        L.tsid_debug_stall_tile_pass.argtypes = [vp, C.c_int64, C.c_int32]
         L.tsid_get_step_times.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_float)]
         L.tsid_sse_noalloc.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
         L.tsid_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
@@ -265,6 +267,11 @@ class Template:
         a, b, c = C.c_int64(0), C.c_int32(0), C.c_int64(0)
         lib().tsid_get_hybrid_info(self.h, C.byref(a), C.byref(b), C.byref(c))
         return a.value, b.value, c.value
+
+    def tsid_debug_stall_tile_pass(self, wait_cycles, item):
+        st = lib().tsid_debug_stall_tile_pass(self.h, int(wait_cycles), int(item))
+        if st != TSID_OK:
+            self._raise(st)
 
     def tsid_set_profiling(self, enable):
         st = lib().tsid_set_profiling(self.h, int(enable))

@@ -237,6 +237,12 @@ tsid_status_t tsid_template_create(const tsid_config_t *cfg, const int32_t *d_ro
     if (bad) { tsid_destroy(t); return fail(nullptr, TSID_ERR_UNSUPPORTED, "TSID_VALUES_U8 promised but a value is not an integer in [0, 255]"); }
   }
   if (path == TSID_PATH_DENSE_TC) {
+    // a dense cell holds one value: a template that lists a cell twice cannot run here (the loss, the counts and
+    // the sparse passes would count both occurrences, the dense matrix only one)
+    int32_t dup = 0;
+    e = csr_has_duplicates(t, &dup);
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+    if (dup) { tsid_destroy(t); return fail(nullptr, TSID_ERR_DUPLICATE, "the dense path cannot hold a (row, col) that occurs twice"); }
     int32_t bad = 0;
     e = dense_build(t, &bad);
     if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
@@ -573,6 +579,16 @@ tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *
     if (t->path == TSID_PATH_HYBRID) *h_launches_per_step = 1 + hybrid_launches_per_step(t) + 1;   // + shadow refresh, update
     else *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? dense_launches_per_step(t) : sparse_launches_per_step(t);
   }
+  return TSID_OK;
+}
+
+tsid_status_t tsid_debug_stall_tile_pass(tsid_template_t *t, int64_t wait_cycles, int32_t item) {
+  if (!t) return TSID_ERR_INVALID_ARG;
+  if (t->path != TSID_PATH_DENSE_TC) return fail(t, TSID_ERR_UNSUPPORTED, "only handles on the dense tensor-core path have bounded waits");
+  if (wait_cycles < 0 || item < 0) return fail(t, TSID_ERR_INVALID_ARG, "wait_cycles and item must be >= 0");
+  t->dbg_wait_cycles = wait_cycles;
+  t->dbg_stall_item = item;
+  fit_graph_release(t);   // a captured graph holds the old launch parameters
   return TSID_OK;
 }
 

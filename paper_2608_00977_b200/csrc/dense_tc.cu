@@ -88,7 +88,8 @@ __global__ void __launch_bounds__(576, 1)
 dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ CUtensorMap tmY,
                   const __grid_constant__ CUtensorMap tmR, int rows_x, int rows_y, int nsplit,
                   float *__restrict__ G, float *__restrict__ Gpart, int32_t *__restrict__ flags,
-                  const DenseChunk *__restrict__ chunks, const int32_t *__restrict__ ylist) {
+                  const DenseChunk *__restrict__ chunks, const int32_t *__restrict__ ylist, long long wait_budget,
+                  int stall_item) {
   using L = Smem<K>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t sm0 = (s32(smem_dyn) + 1023u) & ~1023u;   // tiles need 1024-byte alignment
@@ -144,14 +145,15 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
     if (lane == 0) {
       int jb_next = (ylist && NW > 0) ? __ldg(ylist + t0) : jb0;
       for (int w = 0; w < NW && ok; ++w) {
+        if (w == stall_item) break;   // test hook: the loads of this item and of all later ones are never issued
         const int jb = jb_next, ys = w % L::NSY, rs = w % L::NSR;
         if (w + 1 < NW) jb_next = ylist ? __ldg(ylist + t0 + w + 1) : jb + 1;
-        if (w >= L::NSY) ok = mbar_wait(bar(L::B_YEMPTY + ys), ((w / L::NSY) - 1) & 1);
+        if (w >= L::NSY) ok = mbar_wait(bar(L::B_YEMPTY + ys), ((w / L::NSY) - 1) & 1, wait_budget);
         if (!ok) break;
         mbar_expect_tx(bar(L::B_YFULL + ys), L::Y_BYTES);
         for (int c = 0; c < K / 64; ++c)
           tma_load_2d(sm0 + L::OFF_Y + ys * L::Y_BYTES + c * L::XB, &tmY, bar(L::B_YFULL + ys), c * 64, jb * BLK);
-        if (w >= L::NSR) ok = mbar_wait(bar(L::B_REMPTY + rs), ((w / L::NSR) - 1) & 1);
+        if (w >= L::NSR) ok = mbar_wait(bar(L::B_REMPTY + rs), ((w / L::NSR) - 1) & 1, wait_budget);
         if (!ok) break;
         mbar_expect_tx(bar(L::B_RFULL + rs), L::R_BYTES);
         for (int c = 0; c < 2; ++c) {
@@ -167,7 +169,7 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
       constexpr uint32_t ID1 = idesc_bf16(BLK), ID2 = idesc_bf16(K) | (1u << 16);   // second product: B is MN-major
       auto mma1 = [&](int w) -> bool {
         const int ys = w % L::NSY, b = w & 1;
-        if (!mbar_wait(bar(L::B_YFULL + ys), (w / L::NSY) & 1)) return false;
+        if (!mbar_wait(bar(L::B_YFULL + ys), (w / L::NSY) & 1, wait_budget)) return false;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < K / 16; ++ks) {   // A: 16 factor columns = 8 TMEM columns of the X block
@@ -177,12 +179,12 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
         tc_commit(bar(L::B_SFULL + b));
         return true;
       };
-      ok = mbar_wait(bar(L::B_XFULL), 0);
+      ok = mbar_wait(bar(L::B_XFULL), 0, wait_budget);
       if (ok && NW > 0) ok = mma1(0);
       for (int w = 0; w < NW && ok; ++w) {
         const int ys = w % L::NSY, b = w & 1;
         if (w + 1 < NW) ok = mma1(w + 1);
-        if (ok) ok = mbar_wait(bar(L::B_EFULL + b), (w >> 1) & 1);
+        if (ok) ok = mbar_wait(bar(L::B_EFULL + b), (w >> 1) & 1, wait_budget);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
@@ -225,8 +227,8 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
     }
     for (int w = team; w < NW && ok; w += 2) {
       const int b = w & 1, rs = w % L::NSR;
-      ok = mbar_wait(bar(L::B_RFULL + rs), (w / L::NSR) & 1);                 // R tile has landed
-      if (ok) ok = mbar_wait(bar(L::B_SFULL + b), (w >> 1) & 1);              // S is complete
+      ok = mbar_wait(bar(L::B_RFULL + rs), (w / L::NSR) & 1, wait_budget);                 // R tile has landed
+      if (ok) ok = mbar_wait(bar(L::B_SFULL + b), (w >> 1) & 1, wait_budget);              // S is complete
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -268,7 +270,7 @@ dense_pass_kernel(const __nv_bfloat16 *__restrict__ Xg, const __grid_constant__ 
       if (lane == 0) mbar_arrive(bar(L::B_EFULL + b));
     }
     const bool writer = team == 0 && NW > 0;
-    if (ok && writer) ok = __all_sync(0xffffffffu, mbar_wait(bar(L::B_GFULL), 0));
+    if (ok && writer) ok = __all_sync(0xffffffffu, mbar_wait(bar(L::B_GFULL), 0, wait_budget));
     if (ok && writer) {
       tc_fence_after();
       float *grow = Gout + (size_t)(grow0 + row) * K + h * (K / 2);
@@ -342,11 +344,12 @@ int dense_split(int rows_x, int rows_y) {
 template <int K>
 cudaError_t launch_dense_pass(cudaStream_t st, const __nv_bfloat16 *X, const CUtensorMap &tmY,
                               const CUtensorMap &tmR, int rows_x, int rows_y, float *G, float *Gpart,
-                              int32_t *flags) {
+                              int32_t *flags, long long wait_budget, int stall_item) {
   auto kern = dense_pass_kernel<K>;
   CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<K>::TOTAL));
   const int nrb = rows_x / BLK, nsplit = dense_split(rows_x, rows_y);
-  kern<<<nrb * nsplit, 576, Smem<K>::TOTAL, st>>>(X, tmY, tmR, rows_x, rows_y, nsplit, G, Gpart, flags, nullptr, nullptr);
+  kern<<<nrb * nsplit, 576, Smem<K>::TOTAL, st>>>(X, tmY, tmR, rows_x, rows_y, nsplit, G, Gpart, flags, nullptr, nullptr,
+                                                  wait_budget, stall_item);
   if (nsplit > 1) {
     const size_t n4 = (size_t)rows_x * K / 4;
     add_partials_kernel<<<148 * 4, 256, 0, st>>>(reinterpret_cast<float4 *>(G), reinterpret_cast<const float4 *>(Gpart),
@@ -413,11 +416,11 @@ cudaError_t dense_tiles_pass(cudaStream_t st, int k, const __nv_bfloat16 *X, con
   if (k == 128) {
     auto kern = dense_pass_kernel<128>;
     CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::TOTAL));
-    kern<<<nchunks, 576, Smem<128>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist);
+    kern<<<nchunks, 576, Smem<128>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist, WAIT_CYCLES, -1);
   } else {
     auto kern = dense_pass_kernel<64>;
     CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::TOTAL));
-    kern<<<nchunks, 576, Smem<64>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist);
+    kern<<<nchunks, 576, Smem<64>::TOTAL, st>>>(X, tmY, tmR, 0, 0, 1, nullptr, partial, flags, chunks, ylist, WAIT_CYCLES, -1);
   }
   return cudaGetLastError();
 }
@@ -428,14 +431,16 @@ cudaError_t dense_grad(tsid_template *t, float *GP, float *GQ) {
   const tsid_config_t &c = t->cfg;
   cudaStream_t st = t->stream;
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW0], st);
-  if (c.k == 128) CK(launch_dense_pass<128>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags));
-  else CK(launch_dense_pass<64>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags));
+  const long long wb = t->dbg_wait_cycles > 0 ? t->dbg_wait_cycles : WAIT_CYCLES;
+  const int stall = t->dbg_wait_cycles > 0 ? t->dbg_stall_item : -1;
+  if (c.k == 128) CK(launch_dense_pass<128>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags, wb, stall));
+  else CK(launch_dense_pass<64>(st, t->rowside.shadow, d->tmQ, d->tmR, c.m, c.n, GP, d->gpart, t->flags, wb, stall));
   if (t->prof.on && t->prof.nsteps < kProfSteps) {
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_ROW1], st);
     cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL0], st);
   }
-  if (c.k == 128) CK(launch_dense_pass<128>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags));
-  else CK(launch_dense_pass<64>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags));
+  if (c.k == 128) CK(launch_dense_pass<128>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags, wb, stall));
+  else CK(launch_dense_pass<64>(st, t->colside.shadow, d->tmP, d->tmRT, c.n, c.m, GQ, d->gpart, t->flags, wb, stall));
   if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + EV_COL1], st);
   return cudaSuccess;
 }

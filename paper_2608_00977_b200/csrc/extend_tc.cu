@@ -1,8 +1,8 @@
 // Stage II (Sec. 5.2, Eq. 10), the gradient GEMM fused with the Adam update, on the tensor cores:
 //       G = U Q^T   (chunk columns x template columns, contraction over the rank k)
 //       g = -2 G + 2 lambda C;  Adam update of C and its moments
-// The paper runs Stage II's products in mixed precision (half-precision operands, fp32 accumulation,
-// Sec. 5.2 "batched matrix multiplications ... mixed precision"); this is that variant: U and Q are
+// The paper runs Stage II's products in mixed precision (Sec. 5.2, Tensor Core acceleration of Stage II:
+// half-precision operands, fp32 accumulation); this is that variant: U and Q are
 // rounded to bf16, the products accumulate in fp32 in TMEM, and C and the Adam moments stay fp32.
 //
 // CTA = 128 rows of the chunk (its U block is converted and copied to TMEM once) x a range of

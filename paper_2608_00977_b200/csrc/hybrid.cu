@@ -253,6 +253,22 @@ struct HybridState {
   alignas(64) unsigned char mapPh[128], mapQh[128], mapRA[128], mapRB[128];
 };
 
+// *h_dup = 1 if some (row, col) occurs twice in the CSR arrays (neighbours: the CSR is sorted by column within a row)
+cudaError_t csr_has_duplicates(tsid_template *t, int32_t *h_dup) {
+  cudaStream_t st = t->stream;
+  const int gr = (int)(((int64_t)t->rowside.nseg * 32 + 255) / 256);
+  CK(cudaMemsetAsync(t->flags + FLAG_DUP, 0, sizeof(int32_t), st));
+  if (t->rowside.nseg > 0) {
+    dup_csr_kernel<<<gr, 256, 0, st>>>(t->rowside.segs, t->rowside.nseg, t->col_idx, t->flags);
+    dup_border_kernel<<<grid_for(t->rowside.nseg, 256), 256, 0, st>>>(t->rowside.segs, t->rowside.nseg, t->row_ptr, t->col_idx, t->flags);
+  }
+  CK(cudaGetLastError());
+  CK(cudaMemcpyAsync(h_dup, t->flags + FLAG_DUP, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  if (*h_dup) CK(cudaMemsetAsync(t->flags + FLAG_DUP, 0, sizeof(int32_t), st));
+  return cudaSuccess;
+}
+
 bool hybrid_qualifies(const tsid_config_t &c) {
   if (c.precision != TSID_BF16_SHADOW || (c.k != 64 && c.k != 128)) return false;
   if (c.clip == TSID_CLIP_ASYM_ENTRY || (c.flags & TSID_VALUES_U8)) return false;

@@ -95,6 +95,10 @@ struct tsid_template {
   const float *fit_P, *fit_Q;
   int fit_steps;
   bool fit_graph_off;  // a capture failed once: launch step by step from then on
+  // test hook (tsid_debug_stall_tile_pass): cycle budget of the dense kernel's waits and the work item whose
+  // loads its producer never issues; 0 = normal operation
+  long long dbg_wait_cycles;
+  int dbg_stall_item;
   char err[256];
 };
 
@@ -193,6 +197,7 @@ cudaError_t dense_tiles_pass(cudaStream_t st, int k, const __nv_bfloat16 *X, con
 
 // hybrid path (hybrid.cu): the populated 128 x 128 tiles of the degree-ordered template on the tensor cores,
 // every other entry through the gather-reduce passes
+cudaError_t csr_has_duplicates(tsid_template *t, int32_t *h_dup);
 bool hybrid_qualifies(const tsid_config_t &c);
 HybridState *hybrid_new();
 void hybrid_delete(HybridState *h);

@@ -213,3 +213,35 @@ def test_update_with_the_exchange_folded_in(case, world):
     assert L.tsid_apply_sliced(T.h, Ps[0].data_ptr(), shards[0].GP.data_ptr(), qa, ga, 0, world) == B.TSID_ERR_INVALID_ARG
     for s in shards:
         s.destroy()
+
+
+@pytest.mark.parametrize("precision", ["f32", "bf16"])
+def test_two_processes_step_a_row_sharded_template_over_a_process_group(precision):
+    """RowShard.step with a real process group: two processes (both on this GPU), gloo underneath, three steps,
+    rank 0 checks the assembled factors against the oracle's full-batch steps.  The exchange happens on the host
+    with a bounded timeout; no kernel of one rank waits for the other, and no NVLink multicast is involved."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port),
+                   NCCL_NVLS_ENABLE="0")
+        procs.append(subprocess.Popen([sys.executable, os.path.join(here, "sharded_worker.py"), precision], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+    outs = []
+    for p in procs:
+        try:
+            out, _ = p.communicate(timeout=240)
+        except subprocess.TimeoutExpired:
+            for q in procs:
+                q.kill()
+            raise
+        outs.append(out)
+    assert all(p.returncode == 0 for p in procs), outs
+    assert "replicas_equal True" in outs[0]

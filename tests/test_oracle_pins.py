@@ -420,6 +420,56 @@ def test_bf16_emulation_rounds_inputs_only():
     np.testing.assert_allclose(e, vals - np.sum(Pb[rows].astype(np.float64) * Qb[cols], axis=1), atol=1e-12)
 
 
+def test_fp16_round_table_and_library_cast():
+    with open(__import__("os").path.join(__import__("conftest").ROOT, "tests", "golden", "fp16_rne.txt")) as f:
+        rowsf = [l.split("#")[0].split() for l in f if l.split("#")[0].strip()]
+    assert len(rowsf) >= 15
+    for a, b in rowsf:
+        x = struct.unpack("<f", struct.pack("<I", int(a, 16)))[0]
+        got = struct.unpack("<I", struct.pack("<f", oracle.fp16_round(x)))[0]
+        assert got == int(b, 16), (a, b, hex(got))
+    # and a library's round-to-nearest-even cast on random values over the whole range of a rating matrix
+    rng = np.random.default_rng(3)
+    xs = np.concatenate([rng.normal(0, 3, 2000), rng.uniform(-70000, 70000, 200), rng.normal(0, 1e-6, 200)]).astype(np.float32)
+    with np.errstate(over="ignore"):
+        ref = xs.astype(np.float16).astype(np.float32)
+    got = np.array([oracle.fp16_round(float(x)) for x in xs], dtype=np.float32)
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+def test_tensor_core_emulation_level(golden_3x2):
+    """Level 2 of the emulation switch: r -> binary16, e -> bfloat16 before the gradient products, factors -> bfloat16.
+    A hand-worked value where each rounding decides the result, then dense algebra with library casts."""
+    g = golden_3x2
+    m, n, k, rows, cols, _, P, Q = _inst(g)
+    vals = _arr(g, "vals_tensor", dtype=np.float32)
+    e = oracle.residuals(m, n, k, rows, cols, vals, P, Q, bf16_emulate=oracle.EMU_TENSOR)
+    assert np.array_equal(e, _arr(g, "e_tensor"))
+    st = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, 0.1, 0.25, 2.0, bf16_emulate=oracle.EMU_TENSOR)
+    assert np.array_equal(st.GP, _arr(g, "GP_tensor", (m, k))) and np.array_equal(st.GQ, _arr(g, "GQ_tensor", (n, k)))
+    lvl1 = oracle.grad_step(m, n, k, rows, cols, vals, P, Q, 0.1, 0.25, 2.0, bf16_emulate=True)
+    assert not np.array_equal(lvl1.GP, st.GP)
+    # random instance: E = mask .* bf16(fp16(R) - Pb Qb^T) by numpy on the dense matrix, then two dense products
+    import torch
+    m2, n2, k2, nnz = 37, 29, 16, 500
+    rows, cols, vals, P2, Q2 = _random_instance(m2, n2, k2, nnz, 21)
+    vals = (vals * 3).astype(np.float32)
+    Pb = torch.from_numpy(P2).to(torch.bfloat16).to(torch.float64).numpy()
+    Qb = torch.from_numpy(Q2).to(torch.bfloat16).to(torch.float64).numpy()
+    R16 = np.zeros((m2, n2)); M = np.zeros((m2, n2))
+    R16[rows, cols] = torch.from_numpy(vals).to(torch.float16).to(torch.float64).numpy(); M[rows, cols] = 1
+    E = torch.from_numpy(((R16 - Pb @ Qb.T) * M).astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    st = oracle.grad_step(m2, n2, k2, rows, cols, vals, P2, Q2, 0.05, 0.03, 0.1, 1, 1, 1, bf16_emulate=oracle.EMU_TENSOR)
+    np.testing.assert_allclose(st.GP, E @ Qb, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(st.GQ, E.T @ Pb, rtol=0, atol=1e-12)
+    assert np.max(np.abs(st.GP - oracle.grad_step(m2, n2, k2, rows, cols, vals, P2, Q2, 0.05, 0.03, 0.1, 1, 1, 1,
+                                                  bf16_emulate=True).GP)) > 1e-4      # the level is not a no-op
+    # the update still starts from the fp32 master and regularises with it
+    s = np.maximum(1, np.bincount(rows, minlength=m2))[:, None]
+    D = np.minimum(2 * st.GP / s - 2 * 0.03 * P2.astype(np.float64), 0.1)
+    np.testing.assert_allclose(st.P, (P2 + 0.05 * D).astype(np.float32), rtol=0, atol=1e-7)
+
+
 # ---------------------------------------------------------------- layout
 @pytest.mark.parametrize("m,n,nnz,seed", [(50, 40, 600, 1), (1, 70, 33, 2), (64, 1, 20, 3), (9, 9, 81, 4), (5, 5, 0, 5)])
 def test_layout_against_lexsort_and_invariants(m, n, nnz, seed):
