@@ -29,6 +29,11 @@ def _sampled_check(w, path, tol_g, n_random=4096, n_hot=16, emulate=True, tol_tr
     T.tsid_grad_step(P, Q, GP, GQ)
     T.tsid_check()
     got_path = T.tsid_get_info()[0]
+    # run to run: the sums of a second evaluation at the same factors have the same bits
+    GP2, GQ2 = torch.empty_like(P), torch.empty_like(Q)
+    T.tsid_grad(tpl.P0, tpl.Q0, GP2, GQ2)
+    assert torch.equal(GP2, GP) and torch.equal(GQ2, GQ)
+    del GP2, GQ2
     # global: the trace identity, with the factor values the passes read
     bf = w.precision == "bf16"
     Pr = tpl.P0.bfloat16().double() if bf else tpl.P0.double()
