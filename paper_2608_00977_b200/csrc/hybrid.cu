@@ -91,11 +91,12 @@ __global__ void tile_count_kernel(const Segment *__restrict__ segs, int nseg, co
     atomicAdd(&cnt[rb + jb], 1u);
   }
 }
-// hist[c] = number of tiles that hold exactly c entries (c = 0 .. 16384)
-__global__ void count_hist_kernel(const uint32_t *__restrict__ cnt, int64_t ntile, uint32_t *__restrict__ hist) {
+// hist[c] = number of tiles that hold exactly c entries, for c = minc .. 16384 (the thin tiles, which are most
+// of them and would all hit the same few counters, are of no interest to the threshold search)
+__global__ void count_hist_kernel(const uint32_t *__restrict__ cnt, int64_t ntile, uint32_t minc, uint32_t *__restrict__ hist) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < ntile; i += (int64_t)gridDim.x * blockDim.x) {
     const uint32_t c = cnt[i];
-    if (c > 0) atomicAdd(&hist[c > (uint32_t)HCELLS ? (uint32_t)HCELLS : c], 1u);
+    if (c >= minc) atomicAdd(&hist[c > (uint32_t)HCELLS ? (uint32_t)HCELLS : c], 1u);
   }
 }
 // flagA[ib * JB + jb] = flagB[jb * IB + ib] = tile stored; one extra zero behind each (the scans need it)
@@ -228,7 +229,9 @@ hot_add_kernel(float4 *__restrict__ G, const int32_t *__restrict__ of_rank, int3
 
 int64_t hybrid_max_tiles(const tsid_config_t &c) {
   const int64_t IB = (c.m + HB - 1) / HB, JB = (c.n + HB - 1) / HB;
-  int64_t mt = (int64_t)kBytesPerEntryForTiles * c.nnz / (2 * HCELLS * (int64_t)sizeof(__half));
+  int64_t bpe = kBytesPerEntryForTiles;
+  if (const char *ev = getenv("TSID_HYBRID_TILE_BYTES")) { const long v = atol(ev); if (v >= 1 && v <= 256) bpe = v; }
+  int64_t mt = bpe * c.nnz / (2 * HCELLS * (int64_t)sizeof(__half));
   if (mt > IB * JB) mt = IB * JB;
   if (mt > (1 << 23)) mt = 1 << 23;   // tile row coordinates of the tensor map stay below 2^31
   return mt < 1 ? 1 : mt;
@@ -345,8 +348,10 @@ cudaError_t hybrid_build(tsid_template *t, LayoutScratch &s, int32_t *h_status) 
   CK(cudaMemsetAsync(cnt, 0, sizeof(uint32_t) * (size_t)NT, st));
   tile_count_kernel<<<gr_row, segthreads, 0, st>>>(t->rowside.segs, t->rowside.nseg, t->col_idx, h->rank_of_row,
                                                    h->rank_of_col, JB, cnt);
+  uint32_t minc = kMinTileEntries;
+  if (const char *ev = getenv("TSID_HYBRID_MIN_TILE")) { const long v = atol(ev); if (v >= 1 && v <= HCELLS) minc = (uint32_t)v; }
   CK(cudaMemsetAsync(s.hist, 0, sizeof(uint32_t) * (HCELLS + 1), st));
-  count_hist_kernel<<<grid_for(NT, 256), 256, 0, st>>>(cnt, NT, s.hist);
+  count_hist_kernel<<<grid_for(NT, 256), 256, 0, st>>>(cnt, NT, minc, s.hist);
   CK(cudaGetLastError());
   std::vector<uint32_t> hist(HCELLS + 1);
   int32_t hf[FLAG_COUNT];
@@ -356,8 +361,6 @@ cudaError_t hybrid_build(tsid_template *t, LayoutScratch &s, int32_t *h_status) 
   if (hf[FLAG_DUP]) { CK(cudaMemsetAsync(t->flags + FLAG_DUP, 0, sizeof(int32_t), st)); return cudaSuccess; }
 
   // 3. threshold: at least kMinTileEntries, raised until the stored tiles fit the reserved memory
-  uint32_t minc = kMinTileEntries;
-  if (const char *ev = getenv("TSID_HYBRID_MIN_TILE")) { const long v = atol(ev); if (v >= 1 && v <= HCELLS) minc = (uint32_t)v; }
   int64_t ntl = 0, ent = 0;
   uint32_t thresh = HCELLS + 1;
   for (int cc = HCELLS; cc >= (int)minc; --cc) {
