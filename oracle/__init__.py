@@ -205,3 +205,21 @@ def extend(m, d, k, col_ptr, row_idx, vals, P, Q, eta, lam, iters, C0=None, beta
                     C.c_double(eta), C.c_double(lam), C.c_double(beta1), C.c_double(beta2), C.c_double(eps),
                     C.c_int32(iters), _p(Cm, C.c_double), C.byref(sse))
     return Cm, sse.value
+
+
+def extend_mixed(m, d, k, col_ptr, row_idx, vals, P, Q, eta, lam, iters, C0=None, beta1=0.9, beta2=0.999, eps=1e-8,
+                 round_operands=True):
+    """Stage II with the operands of its two products rounded to bfloat16 (the paper's mixed precision, Sec. 5.2).
+    round_operands=False is the same iteration in full precision.  Returns (C float64 [ncols, d], sse)."""
+    col_ptr = np.ascontiguousarray(col_ptr, dtype=np.int64)
+    row_idx = np.ascontiguousarray(row_idx, dtype=np.int32)
+    vals = np.ascontiguousarray(vals, dtype=np.float32)
+    ncols = col_ptr.shape[0] - 1
+    P, Q = _fac(P, m, k), _fac(Q, d, k)
+    Cm = np.zeros((ncols, d), dtype=np.float64) if C0 is None else np.ascontiguousarray(C0, dtype=np.float64).copy()
+    sse = C.c_double(0.0)
+    _L().orc_extend_mixed(C.c_int32(m), C.c_int32(d), C.c_int32(k), C.c_int32(ncols), _p(col_ptr, C.c_int64),
+                          _p(row_idx, C.c_int32), _p(vals, C.c_float), _p(P, C.c_float), _p(Q, C.c_float),
+                          C.c_double(eta), C.c_double(lam), C.c_double(beta1), C.c_double(beta2), C.c_double(eps),
+                          C.c_int32(iters), C.c_int(int(round_operands)), _p(Cm, C.c_double), C.byref(sse))
+    return Cm, sse.value

@@ -433,3 +433,63 @@ void orc_extend(int32_t m, int32_t d, int32_t k, int32_t ncols, const int64_t *c
   if (sse_out) *sse_out = sse;
   free(Rhat); free(g); free(mo); free(vo);
 }
+
+/* Stage II in the paper's mixed precision (Sec. 5.2: the products of Stage II run with half-precision operands
+ * and fp32 accumulation).  The same Adam iteration as orc_extend, but written in the factored form in which the
+ * mixed-precision products appear, with the operands of exactly those two products rounded to bfloat16 (nearest
+ * even) and every sum exact:
+ *       W_j = Q^T bf(C_j)            first product   (k values: Rhat*_i C_j = p_i . W_j)
+ *       e_i = R_ij - p_i . W_j ,  U_j = sum_i e_i p_i                         (full precision)
+ *       g   = -2 bf(Q) bf(U_j) + 2 lambda C_j       second product
+ * bf(.) = bfloat16 rounding; Q is rounded in both products; C, the Adam moments, the residuals and U stay in
+ * full precision (C is rounded only where it enters the first product; it is first taken to fp32, the precision
+ * the stored coefficients have).  With rounding switched off this is orc_extend re-associated, which is how it is
+ * pinned (besides dense algebra with library casts for where the rounding sits). */
+void orc_extend_mixed(int32_t m, int32_t d, int32_t k, int32_t ncols, const int64_t *col_ptr,
+                      const int32_t *row_idx, const float *vals, const float *P, const float *Q,
+                      double eta, double lambda, double b1, double b2, double eps, int32_t iters,
+                      int round_operands, double *C, double *sse_out) {
+  (void)m;
+  double *Qr = (double *)malloc(sizeof(double) * (size_t)d * k);
+  for (size_t a = 0; a < (size_t)d * k; ++a) Qr[a] = round_operands ? (double)orc_bf16_round(Q[a]) : (double)Q[a];
+  double *W = (double *)malloc(sizeof(double) * (size_t)k);
+  double *U = (double *)malloc(sizeof(double) * (size_t)k);
+  double *mo = (double *)malloc(sizeof(double) * (size_t)d);
+  double *vo = (double *)malloc(sizeof(double) * (size_t)d);
+  double sse = 0.0;
+  for (int32_t j = 0; j < ncols; ++j) {
+    double *Cj = C + (size_t)j * d;
+    for (int32_t a = 0; a < d; ++a) { mo[a] = 0.0; vo[a] = 0.0; }
+    double p1 = 1.0, p2 = 1.0;
+    for (int32_t it = 1; it <= iters + 1; ++it) {          /* the extra round only evaluates the SSE */
+      for (int32_t l = 0; l < k; ++l) W[l] = 0.0;
+      for (int32_t a = 0; a < d; ++a) {
+        double c = round_operands ? (double)orc_bf16_round((float)Cj[a]) : Cj[a];
+        for (int32_t l = 0; l < k; ++l) W[l] += c * Qr[(size_t)a * k + l];
+      }
+      for (int32_t l = 0; l < k; ++l) U[l] = 0.0;
+      for (int64_t t = col_ptr[j]; t < col_ptr[j + 1]; ++t) {
+        const float *pi = P + (size_t)row_idx[t] * k;
+        double pred = 0.0;
+        for (int32_t l = 0; l < k; ++l) pred += (double)pi[l] * W[l];
+        double e = (double)vals[t] - pred;
+        if (it > iters) sse += e * e;
+        for (int32_t l = 0; l < k; ++l) U[l] += e * (double)pi[l];
+      }
+      if (it > iters) break;
+      if (round_operands) for (int32_t l = 0; l < k; ++l) U[l] = (double)orc_bf16_round((float)U[l]);
+      p1 *= b1; p2 *= b2;
+      for (int32_t a = 0; a < d; ++a) {
+        double qu = 0.0;
+        for (int32_t l = 0; l < k; ++l) qu += Qr[(size_t)a * k + l] * U[l];
+        double g = -2.0 * qu + 2.0 * lambda * Cj[a];
+        mo[a] = b1 * mo[a] + (1.0 - b1) * g;
+        vo[a] = b2 * vo[a] + (1.0 - b2) * g * g;
+        double mh = mo[a] / (1.0 - p1), vh = vo[a] / (1.0 - p2);
+        Cj[a] -= eta * mh / (sqrt(vh) + eps);
+      }
+    }
+  }
+  if (sse_out) *sse_out = sse;
+  free(Qr); free(W); free(U); free(mo); free(vo);
+}

@@ -98,3 +98,40 @@ def test_columns_are_independent_and_warm_start_continues():
             fd = (_loss_col(Rhat, rows, r, cp_, 0.1) - _loss_col(Rhat, rows, r, cm_, 0.1)) / (2 * h)
             step = C1[j, a] - C0[j, a]
             np.testing.assert_allclose(step, -1e-3 * fd / (abs(fd) + 1e-8), rtol=1e-5, atol=1e-12)
+
+
+def test_mixed_precision_form_is_the_same_iteration_and_rounds_only_the_product_operands():
+    """orc_extend_mixed: without rounding it is orc_extend re-associated (pinned above against torch's Adam); with
+    rounding, the two places where a bfloat16 value enters are checked by dense algebra with a library's casts."""
+    m, d, k, cp, ri, v, P, Q = _problem(m=40, d=9, k=4, ncols=6, seed=5)
+    rng = np.random.default_rng(1)
+    C0 = (rng.standard_normal((len(cp) - 1, d)) * 0.3).astype(np.float32)
+    for c0 in (None, C0):
+        a, sa = oracle.extend(m, d, k, cp, ri, v, P, Q, 0.03, 0.05, 12, C0=c0)
+        b, sb = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, 0.03, 0.05, 12, C0=c0, round_operands=False)
+        np.testing.assert_allclose(b, a, rtol=1e-9, atol=1e-12)
+        assert abs(sa - sb) <= 1e-9 * sa
+
+    def bf(x):
+        return torch.tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    Qb, Pd = bf(Q), P.astype(np.float64)
+    # one step with eps so large that the step is -eta g / eps: reads off the gradient, from a warm start
+    eta, lam, eps = 1.0, 0.05, 1e6
+    C1, _ = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, eta, lam, 1, C0=C0, eps=eps)
+    for j in range(len(cp) - 1):
+        rows, r = ri[cp[j]:cp[j + 1]], v[cp[j]:cp[j + 1]].astype(np.float64)
+        W = Qb.T @ bf(C0[j])                               # first product: both operands rounded
+        e = r - Pd[rows] @ W                               # residuals in full precision
+        U = Pd[rows].T @ e
+        g = -2 * Qb @ bf(U) + 2 * lam * C0[j].astype(np.float64)    # second product: both operands rounded, C itself not
+        np.testing.assert_allclose(C1[j] - C0[j], -eta * g / (np.abs(g) + eps), rtol=1e-9, atol=1e-15)
+    # and the rounding is not a no-op on these inputs
+    C1f, _ = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, eta, lam, 1, C0=C0, eps=eps, round_operands=False)
+    assert np.max(np.abs(C1f - C1)) > 1e-3 * np.max(np.abs(C1 - C0))
+    # the SSE it reports is that of the rounded first product at the returned coefficients
+    C2, sse = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, 0.03, lam, 5)
+    tot = 0.0
+    for j in range(len(cp) - 1):
+        rows, r = ri[cp[j]:cp[j + 1]], v[cp[j]:cp[j + 1]].astype(np.float64)
+        tot += float(np.sum((r - Pd[rows] @ (Qb.T @ bf(C2[j]))) ** 2))
+    assert abs(tot - sse) <= 1e-9 * sse

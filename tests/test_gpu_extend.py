@@ -148,8 +148,47 @@ def test_extend_tensor_core_form(m, d, k, ncols, per_col, chunk):
     assert rms <= 0.1, rms
     assert abs(sse_tc - sse_r) / sse_r <= 1e-3
     assert not C_tc[min(3, ncols - 1)].any()
+    # (3) element by element against the oracle that rounds the operands of the two products as this form does
+    # (the loose bounds above compare a bf16 computation with an fp64 one; here only fp32 summation is left, plus
+    # Adam's sensitivity on coordinates whose gradient nearly cancels, which the fp32 form has as well)
+    # One thing besides summation order is left: a coordinate of U that sits within fp32 rounding of the midpoint of
+    # two bf16 values rounds the other way in the kernel (about 1 in 10^4); that moves the whole gradient of its column
+    # by one bf16 step of that coordinate times a row of Q.  So: all but a few columns within 1e-5, none further off
+    # than two such flips.
+    colof = np.repeat(np.arange(ncols), np.diff(cp))
+    U0 = np.zeros((ncols, k)); np.add.at(U0, colof, v[:, None].astype(np.float64) * P[ri].astype(np.float64))
+    flip = 2.0 * 2.0 ** -8 * np.abs(U0).max() * np.abs(Q).max() * (1.0 / 1e4)      # in units of the step: eta / eps = 1e-4
+    for c0 in (None, C0):
+        Ch.zero_() if c0 is None else Ch.copy_(torch.tensor(c0))
+        B.tsid_extend(*args, Ch, chunk, 1, 1.0, 0.05, eps=1e4, tensor_cores=True)
+        Cm, _ = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, 1.0, 0.05, 1, C0=c0, eps=1e4)
+        base = 0.0 if c0 is None else c0
+        err = np.abs((Ch.numpy() - base) - (Cm - base))
+        loose = err > 1e-5 * np.max(np.abs(Cm - base))
+        assert loose.any(axis=1).mean() <= 0.03 and err.max() <= 2 * 2 * flip, (loose.any(axis=1).mean(), err.max(), flip)
+    Cm, sse_m = oracle.extend_mixed(m, d, k, cp, ri, v, P, Q, eta, lam, iters)
+    scale = float(np.abs(Cm).max())
+    err = np.abs(C_tc - Cm)
+    assert abs(sse_tc - sse_m) <= 1e-4 * sse_m, (sse_tc, sse_m)
+    assert float(np.sqrt(np.mean(err ** 2))) <= 1e-3 * scale and int((err > 2e-3 * scale).sum()) <= max(3, err.size // 2000), (
+        float(np.sqrt(np.mean(err ** 2))) / scale, int((err > 2e-3 * scale).sum()), err.size)
     # a shape the tensor-core form does not take is refused, not silently run another way
     with pytest.raises(B.TsidError) as e:
         B.tsid_extend(torch.tensor(P[:, :32].copy(), device=DEV), torch.tensor(Q[:, :32].copy(), device=DEV), *args[2:], Ch,
                       chunk, 1, eta, lam, tensor_cores=True)
     assert e.value.status == B.TSID_ERR_UNSUPPORTED
+
+
+def test_extend_tensor_core_form_refuses_a_width_it_cannot_tile():
+    """d must be a multiple of 8 (16-byte rows of the bf16 copy, a TMA requirement): 260 is refused, not padded."""
+    P, Q, cp, ri, v = _problem(300, 260, 64, 40, 30, seed=2)
+    Ch = torch.zeros(40, 260).pin_memory()
+    with pytest.raises(B.TsidError) as e:
+        B.tsid_extend(torch.tensor(P, device=DEV), torch.tensor(Q, device=DEV), torch.tensor(cp).pin_memory(),
+                      torch.tensor(ri).pin_memory(), torch.tensor(v).pin_memory(), Ch, 20, 2, 0.02, 0.05, tensor_cores=True)
+    assert e.value.status == B.TSID_ERR_UNSUPPORTED
+    # the fp32 form takes the same shape
+    B.tsid_extend(torch.tensor(P, device=DEV), torch.tensor(Q, device=DEV), torch.tensor(cp).pin_memory(),
+                  torch.tensor(ri).pin_memory(), torch.tensor(v).pin_memory(), Ch, 20, 2, 0.02, 0.05)
+    Cr, _ = oracle.extend(300, 260, 64, cp, ri, v, P, Q, 0.02, 0.05, 2)
+    assert relerr(Ch.numpy(), Cr) <= 2e-3
