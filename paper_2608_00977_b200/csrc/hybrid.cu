@@ -10,7 +10,6 @@
 // in chunk order).  No floating-point atomics; integer atomics only in the tile histogram, whose result
 // does not depend on their order.
 #include <cuda_fp16.h>
-#include <stdlib.h>
 
 #include <new>
 #include <vector>
@@ -229,9 +228,7 @@ hot_add_kernel(float4 *__restrict__ G, const int32_t *__restrict__ of_rank, int3
 
 int64_t hybrid_max_tiles(const tsid_config_t &c) {
   const int64_t IB = (c.m + HB - 1) / HB, JB = (c.n + HB - 1) / HB;
-  int64_t bpe = kBytesPerEntryForTiles;
-  if (const char *ev = getenv("TSID_HYBRID_TILE_BYTES")) { const long v = atol(ev); if (v >= 1 && v <= 256) bpe = v; }
-  int64_t mt = bpe * c.nnz / (2 * HCELLS * (int64_t)sizeof(__half));
+  int64_t mt = (int64_t)kBytesPerEntryForTiles * c.nnz / (2 * HCELLS * (int64_t)sizeof(__half));
   if (mt > IB * JB) mt = IB * JB;
   if (mt > (1 << 23)) mt = 1 << 23;   // tile row coordinates of the tensor map stay below 2^31
   return mt < 1 ? 1 : mt;
@@ -348,8 +345,7 @@ cudaError_t hybrid_build(tsid_template *t, LayoutScratch &s, int32_t *h_status) 
   CK(cudaMemsetAsync(cnt, 0, sizeof(uint32_t) * (size_t)NT, st));
   tile_count_kernel<<<gr_row, segthreads, 0, st>>>(t->rowside.segs, t->rowside.nseg, t->col_idx, h->rank_of_row,
                                                    h->rank_of_col, JB, cnt);
-  uint32_t minc = kMinTileEntries;
-  if (const char *ev = getenv("TSID_HYBRID_MIN_TILE")) { const long v = atol(ev); if (v >= 1 && v <= HCELLS) minc = (uint32_t)v; }
+  const uint32_t minc = kMinTileEntries;
   CK(cudaMemsetAsync(s.hist, 0, sizeof(uint32_t) * (HCELLS + 1), st));
   count_hist_kernel<<<grid_for(NT, 256), 256, 0, st>>>(cnt, NT, minc, s.hist);
   CK(cudaGetLastError());
