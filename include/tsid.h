@@ -248,6 +248,23 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
  * tsid_grad_step launches. */
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
 
+/* Mini-batch form (Sec. 5.1: the updates run over mini-batches of observed entries, aggregated per factor row and divided
+ * by the number of contributors, Eq. 9; a mini-batch step is the full-batch step above restricted to the batch's entries,
+ * with Eq. 9's n counted inside the batch).  ONE template holds all batches: d_batch (DEVICE, int32[nnz]) gives the batch of
+ * every COO triple, 0 <= batch < n_batches; the layout pass sorts by (batch, row, col) and (batch, col, row) in one go, so
+ * every batch owns a contiguous range of work segments in one workspace (tsid_workspace_bytes_batched bytes).  cfg.m, cfg.n
+ * are the sizes of P and Q as usual.  tsid_grad_step_batch runs one step on batch `batch` (the other arguments as in
+ * tsid_grad_step; the raw sums returned are those of the batch); an epoch is one call per batch, in the caller's order.
+ * Sparse path only (cfg.path AUTO or SPARSE), fp32 value streams, n_batches * m and n_batches * n below 2^31,
+ * n_batches <= 65536.  The other stepping, loss and count calls refuse such a handle (TSID_ERR_UNSUPPORTED).
+ * Errors: as tsid_template_create; TSID_ERR_INDEX_RANGE also for a batch number out of range. */
+tsid_status_t tsid_workspace_bytes_batched(const tsid_config_t *cfg, int32_t n_batches, size_t *h_bytes_out);
+tsid_status_t tsid_template_create_batched(const tsid_config_t *cfg, const int32_t *d_rows, const int32_t *d_cols,
+                                           const float *d_vals, const int32_t *d_batch, int32_t n_batches,
+                                           tsid_template_t **out);
+tsid_status_t tsid_grad_step_batch(tsid_template_t *t, int32_t batch, float *d_P, float *d_Q, float *d_gradP_or_null,
+                                   float *d_gradQ_or_null);
+
 /* What the hybrid path stored (debug / bench surface): the number of 128 x 128 tiles kept densely, the
  * smallest number of entries such a tile holds, and how many entries stayed on the gather-reduce passes.
  * On a handle of another path all three are 0 (tail = nnz).  Any out pointer may be NULL. */

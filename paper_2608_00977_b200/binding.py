@@ -34,7 +34,8 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
            "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info", "tsid_get_step_times",
-           "tsid_debug_stall_tile_pass"]
+           "tsid_debug_stall_tile_pass", "tsid_workspace_bytes_batched", "tsid_template_create_batched",
+           "tsid_grad_step_batch"]
 
 
 class TsidConfig(C.Structure):
@@ -94,6 +95,9 @@ def lib():
         L.tsid_set_profiling.argtypes = [vp, C.c_int32]
         L.tsid_get_pass_times.argtypes = [vp, C.POINTER(C.c_int32)] + [C.POINTER(C.c_float)] * 3
         L.tsid_debug_stall_tile_pass.argtypes = [vp, C.c_int64, C.c_int32]
+        L.tsid_workspace_bytes_batched.argtypes = [C.POINTER(TsidConfig), C.c_int32, C.POINTER(C.c_size_t)]
+        L.tsid_template_create_batched.argtypes = [C.POINTER(TsidConfig), vp, vp, vp, vp, C.c_int32, C.POINTER(vp)]
+        L.tsid_grad_step_batch.argtypes = [vp, C.c_int32, vp, vp, vp, vp]
         L.tsid_get_step_times.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_float)]
         L.tsid_sse_noalloc.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
         L.tsid_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.POINTER(C.c_size_t)]
@@ -132,15 +136,27 @@ class Template:
     """Owns the workspace tensor and the handle of one template (tsid_template_create ... tsid_destroy)."""
 
     def __init__(self, cfg: TsidConfig, rows: torch.Tensor, cols: torch.Tensor, vals: torch.Tensor,
-                 stream: torch.cuda.Stream | None = None):
+                 stream: torch.cuda.Stream | None = None, batch: torch.Tensor | None = None, n_batches: int = 0):
+        """batch / n_batches given: a mini-batch template (tsid_template_create_batched), stepped with
+        tsid_grad_step_batch."""
         L = lib()
         nnz = int(cfg.nnz)
+        if batch is not None:
+            _check_tensor(batch, torch.int32, nnz, "batch")
         _check_tensor(rows, torch.int32, nnz, "rows")
         _check_tensor(cols, torch.int32, nnz, "cols")
         _check_tensor(vals, torch.float32, nnz, "vals")
         self.device = rows.device
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
-        need = tsid_workspace_bytes(cfg)
+        if batch is None:
+            need = tsid_workspace_bytes(cfg)
+        else:
+            out = C.c_size_t(0)
+            st = L.tsid_workspace_bytes_batched(C.byref(cfg), int(n_batches), C.byref(out))
+            if st != TSID_OK:
+                raise TsidError(st, L.tsid_last_error(None).decode())
+            need = out.value
+        self.n_batches = int(n_batches) if batch is not None else 0
         self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
         base = (self.workspace.data_ptr() + 255) & ~255
         self.cfg = TsidConfig.from_buffer_copy(cfg)
@@ -150,8 +166,12 @@ class Template:
         self.m, self.n, self.k, self.nnz = int(cfg.m), int(cfg.n), int(cfg.k), nnz
         h = C.c_void_p(None)
         with torch.cuda.device(self.device):
-            st = L.tsid_template_create(C.byref(self.cfg), rows.data_ptr(), cols.data_ptr(), vals.data_ptr(),
-                                        C.byref(h))
+            if batch is None:
+                st = L.tsid_template_create(C.byref(self.cfg), rows.data_ptr(), cols.data_ptr(), vals.data_ptr(),
+                                            C.byref(h))
+            else:
+                st = L.tsid_template_create_batched(C.byref(self.cfg), rows.data_ptr(), cols.data_ptr(), vals.data_ptr(),
+                                                    batch.data_ptr(), int(n_batches), C.byref(h))
         if st != TSID_OK:
             self.h = None
             raise TsidError(st, L.tsid_last_error(None).decode())
@@ -174,6 +194,14 @@ class Template:
         st = lib().tsid_grad_step(self.h, P.data_ptr(), Q.data_ptr(),
                                   gradP.data_ptr() if gradP is not None else None,
                                   gradQ.data_ptr() if gradQ is not None else None)
+        if st != TSID_OK:
+            self._raise(st)
+
+    def tsid_grad_step_batch(self, batch, P, Q, gradP=None, gradQ=None):
+        self._factors(P, Q)
+        st = lib().tsid_grad_step_batch(self.h, int(batch), P.data_ptr(), Q.data_ptr(),
+                                        gradP.data_ptr() if gradP is not None else None,
+                                        gradQ.data_ptr() if gradQ is not None else None)
         if st != TSID_OK:
             self._raise(st)
 

@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/tsid.h: argument checks, workspace carving,
 // and the order of kernel launches of each entry point.  No device allocation happens here.
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "tsid_internal.cuh"
@@ -52,11 +53,14 @@ int resolve_path(const tsid_config_t &c) {
 
 // Carves (or, with a null base, measures) every device buffer of a template.
 void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScratch &ls) {
-  const size_t nnz = (size_t)c.nnz, m = (size_t)c.m, n = (size_t)c.n, k = (size_t)c.k;
+  const size_t nnz = (size_t)c.nnz, k = (size_t)c.k;
+  const size_t mr = (size_t)c.m, nr = (size_t)c.n;                       // sizes of the factor matrices
+  const size_t m = t->vm ? (size_t)t->vm : mr, n = t->vn ? (size_t)t->vn : nr;   // sizes of the layout (virtual for mini-batches)
   const size_t nz = nnz ? nnz : 1;
   t->flags = cv.take<int32_t>(FLAG_COUNT);
   t->row_ptr = cv.take<int64_t>(m + 1);
   t->col_ptr = cv.take<int64_t>(n + 1);
+  if (t->n_batches) { t->vrows = cv.take<int32_t>(nz); t->vcols = cv.take<int32_t>(nz); }
   t->col_idx = cv.take<int32_t>(nz);
   t->val_csr = cv.take<float>(nz);
   t->row_idx = cv.take<int32_t>(nz);
@@ -73,8 +77,9 @@ void carve_all(tsid_template *t, const tsid_config_t &c, Carver &cv, LayoutScrat
     sd.segs = cv.take<Segment>(sd.cap_seg);
     sd.splits = cv.take<SplitRow>(sd.cap_split);
     sd.scale = cv.take<float>(sd.nrows);
-    sd.G = cv.take<float>((size_t)sd.nrows * k);
-    sd.shadow = c.precision == TSID_BF16_SHADOW ? cv.take<__nv_bfloat16>((size_t)sd.nrows * k) : nullptr;
+    const size_t real_rows = i == 0 ? mr : nr;
+    sd.G = cv.take<float>(real_rows * k);
+    sd.shadow = c.precision == TSID_BF16_SHADOW ? cv.take<__nv_bfloat16>(real_rows * k) : nullptr;
   }
   t->rowside.ptr = t->row_ptr; t->rowside.idx = t->col_idx; t->rowside.val = t->val_csr;
   t->colside.ptr = t->col_ptr; t->colside.idx = t->row_idx; t->colside.val = t->val_csc;
@@ -155,8 +160,10 @@ cudaError_t fit_graph_get(tsid_template *t, float *P, float *Q, int steps) {
   return cudaSuccess;
 }
 
-tsid_status_t check_factors(tsid_template *t, const float *P, const float *Q) {
+tsid_status_t check_factors(tsid_template *t, const float *P, const float *Q, bool batch_call = false) {
   if (!t) return TSID_ERR_INVALID_ARG;
+  if (t->n_batches && !batch_call)
+    return fail(t, TSID_ERR_UNSUPPORTED, "a mini-batch template is stepped with tsid_grad_step_batch only");
   if (!P || !Q) return fail(t, TSID_ERR_INVALID_ARG, "P or Q is null");
   if (!aligned16(P) || !aligned16(Q)) return fail(t, TSID_ERR_INVALID_ARG, "P and Q must be 16-byte aligned");
   return TSID_OK;
@@ -295,6 +302,7 @@ tsid_status_t tsid_apply(tsid_template_t *t, float *d_P, float *d_Q, const float
 tsid_status_t tsid_apply_sliced(tsid_template_t *t, float *d_P, const float *d_GP, float *const *h_Q_replicas,
                                 const float *const *h_GQ_parts, int32_t rank, int32_t world) {
   if (!t) return TSID_ERR_INVALID_ARG;
+  if (t->n_batches) return fail(t, TSID_ERR_UNSUPPORTED, "not for a mini-batch template");
   if (!d_P || !d_GP || !h_Q_replicas || !h_GQ_parts || !aligned16(d_P) || !aligned16(d_GP))
     return fail(t, TSID_ERR_INVALID_ARG, "P, G_P and the pointer arrays must be non-null (P, G_P 16-byte aligned)");
   if (world < 1 || world > kMaxRanks || rank < 0 || rank >= world)
@@ -308,6 +316,7 @@ tsid_status_t tsid_apply_sliced(tsid_template_t *t, float *d_P, const float *d_G
 
 tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int32_t *d_cnt_q_or_null) {
   if (!t) return TSID_ERR_INVALID_ARG;
+  if (t->n_batches) return fail(t, TSID_ERR_UNSUPPORTED, "not for a mini-batch template");
   cudaError_t e = cudaSuccess;
   if (d_cnt_p_or_null) e = sparse_counts(t, t->rowside, d_cnt_p_or_null);
   if (e == cudaSuccess && d_cnt_q_or_null) e = sparse_counts(t, t->colside, d_cnt_q_or_null);
@@ -316,6 +325,7 @@ tsid_status_t tsid_get_counts(tsid_template_t *t, int32_t *d_cnt_p_or_null, int3
 
 tsid_status_t tsid_set_norm_counts(tsid_template_t *t, const int32_t *d_cnt_p_or_null, const int32_t *d_cnt_q_or_null) {
   if (!t) return TSID_ERR_INVALID_ARG;
+  if (t->n_batches) return fail(t, TSID_ERR_UNSUPPORTED, "not for a mini-batch template");
   cudaError_t e = cudaSuccess;
   if (d_cnt_p_or_null) e = sparse_scale_from_counts(t, t->rowside, t->cfg.norm_p, d_cnt_p_or_null);
   if (e == cudaSuccess && d_cnt_q_or_null) e = sparse_scale_from_counts(t, t->colside, t->cfg.norm_q, d_cnt_q_or_null);
@@ -415,7 +425,7 @@ static void prof_release(tsid_template *t) {
 }
 
 tsid_status_t tsid_destroy(tsid_template_t *t) {
-  if (t) { prof_release(t); fit_graph_release(t); dense_delete(t->dense); hybrid_delete(t->hybrid); }
+  if (t) { prof_release(t); fit_graph_release(t); dense_delete(t->dense); hybrid_delete(t->hybrid); free(t->bseg_row); }
   delete t;
   return TSID_OK;
 }
@@ -590,6 +600,93 @@ tsid_status_t tsid_debug_stall_tile_pass(tsid_template_t *t, int64_t wait_cycles
   t->dbg_stall_item = item;
   fit_graph_release(t);   // a captured graph holds the old launch parameters
   return TSID_OK;
+}
+
+// ---- mini-batch template -----------------------------------------------------------------------------
+static tsid_status_t check_batched(const tsid_config_t *cfg, int32_t n_batches, char *err) {
+  tsid_status_t st = check_cfg(cfg, err);
+  if (st != TSID_OK) return st;
+  if (n_batches < 1 || n_batches > 65536) { snprintf(err, 256, "n_batches must be in [1, 65536]"); return TSID_ERR_INVALID_ARG; }
+  if (cfg->path == TSID_PATH_DENSE_TC || cfg->path == TSID_PATH_HYBRID || (cfg->flags & TSID_VALUES_U8)) {
+    snprintf(err, 256, "a mini-batch template runs the sparse path with fp32 value streams");
+    return TSID_ERR_UNSUPPORTED;
+  }
+  if ((int64_t)cfg->m * n_batches > 2147483647LL || (int64_t)cfg->n * n_batches > 2147483647LL) {
+    snprintf(err, 256, "n_batches * m and n_batches * n must stay below 2^31");
+    return TSID_ERR_UNSUPPORTED;
+  }
+  return TSID_OK;
+}
+
+tsid_status_t tsid_workspace_bytes_batched(const tsid_config_t *cfg, int32_t n_batches, size_t *h_bytes_out) {
+  if (!h_bytes_out) return fail(nullptr, TSID_ERR_INVALID_ARG, "bytes_out is null");
+  tsid_status_t st = check_batched(cfg, n_batches, g_create_err);
+  if (st != TSID_OK) return st;
+  tsid_template tmp;
+  memset(static_cast<void *>(&tmp), 0, sizeof(tmp));
+  tmp.path = TSID_PATH_SPARSE;
+  tmp.n_batches = n_batches; tmp.vm = cfg->m * n_batches; tmp.vn = cfg->n * n_batches;
+  Carver cv(nullptr);
+  LayoutScratch ls;
+  carve_all(&tmp, *cfg, cv, ls);
+  *h_bytes_out = cv.off;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_template_create_batched(const tsid_config_t *cfg, const int32_t *d_rows, const int32_t *d_cols,
+                                           const float *d_vals, const int32_t *d_batch, int32_t n_batches,
+                                           tsid_template_t **out) {
+  if (!out) return fail(nullptr, TSID_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  tsid_status_t st = check_batched(cfg, n_batches, g_create_err);
+  if (st != TSID_OK) return st;
+  if (cfg->nnz > 0 && (!d_rows || !d_cols || !d_vals || !d_batch)) return fail(nullptr, TSID_ERR_INVALID_ARG, "COO or batch pointer is null");
+  if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255u))
+    return fail(nullptr, TSID_ERR_INVALID_ARG, "workspace is null or not 256-byte aligned");
+  size_t need = 0;
+  tsid_workspace_bytes_batched(cfg, n_batches, &need);
+  if (cfg->workspace_bytes < need) return fail(nullptr, TSID_ERR_OOM, "workspace smaller than tsid_workspace_bytes_batched");
+  tsid_template *t = new (std::nothrow) tsid_template;
+  int32_t *hb = static_cast<int32_t *>(malloc(sizeof(int32_t) * 4 * ((size_t)n_batches + 1)));
+  if (!t || !hb) { delete t; free(hb); return fail(nullptr, TSID_ERR_OOM, "host allocation failed"); }
+  memset(static_cast<void *>(t), 0, sizeof(*t));
+  t->cfg = *cfg;
+  t->cfg.flags &= ~(uint32_t)TSID_INPUT_ROW_SORTED;   // the promise is about (row, col); the layout sorts (batch, row, col)
+  t->stream = static_cast<cudaStream_t>(cfg->stream);
+  t->path = TSID_PATH_SPARSE;
+  t->n_batches = n_batches; t->vm = cfg->m * n_batches; t->vn = cfg->n * n_batches;
+  t->bseg_row = hb; t->bseg_col = hb + (n_batches + 1); t->bsplit_row = hb + 2 * (n_batches + 1); t->bsplit_col = hb + 3 * (n_batches + 1);
+  Carver cv(cfg->workspace);
+  LayoutScratch ls;
+  carve_all(t, t->cfg, cv, ls);
+  int32_t hf[FLAG_COUNT] = {0};
+  cudaError_t e = batch_virtual_coo(t, d_rows, d_cols, d_batch);
+  if (e == cudaSuccess) e = layout_build(t, t->vrows, t->vcols, d_vals, ls, hf);
+  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+  if (hf[FLAG_RANGE]) { tsid_destroy(t); return fail(nullptr, TSID_ERR_INDEX_RANGE, "a row, column or batch index is out of range"); }
+  if (hf[FLAG_DUP] && (cfg->flags & TSID_VALIDATE)) { tsid_destroy(t); return fail(nullptr, TSID_ERR_DUPLICATE, "duplicate (batch, row, col)"); }
+  e = build_segments(t, t->rowside, cfg->norm_p, ls);
+  if (e == cudaSuccess) e = batch_ranges(t, ls, false);
+  if (e == cudaSuccess) e = build_segments(t, t->colside, cfg->norm_q, ls);
+  if (e == cudaSuccess) e = batch_ranges(t, ls, true);
+  if (e != cudaSuccess) { st = cuda_fail(nullptr, e); tsid_destroy(t); return st; }
+  snprintf(t->err, 256, "ok");
+  *out = t;
+  return TSID_OK;
+}
+
+tsid_status_t tsid_grad_step_batch(tsid_template_t *t, int32_t batch, float *d_P, float *d_Q, float *d_gradP_or_null,
+                                   float *d_gradQ_or_null) {
+  tsid_status_t st = check_factors(t, d_P, d_Q, true);
+  if (st != TSID_OK) return st;
+  if (!t->n_batches) return fail(t, TSID_ERR_UNSUPPORTED, "not a mini-batch template");
+  if (batch < 0 || batch >= t->n_batches) return fail(t, TSID_ERR_INVALID_ARG, "batch out of range");
+  if ((d_gradP_or_null && !aligned16(d_gradP_or_null)) || (d_gradQ_or_null && !aligned16(d_gradQ_or_null)))
+    return fail(t, TSID_ERR_INVALID_ARG, "gradient outputs must be 16-byte aligned");
+  float *GP = d_gradP_or_null ? d_gradP_or_null : t->rowside.G;
+  float *GQ = d_gradQ_or_null ? d_gradQ_or_null : t->colside.G;
+  cudaError_t e = sparse_batch_step(t, batch, d_P, d_Q, GP, GQ);
+  return e == cudaSuccess ? TSID_OK : cuda_fail(t, e);
 }
 
 tsid_status_t tsid_get_hybrid_info(const tsid_template_t *t, int64_t *h_tiles, int32_t *h_min_tile_entries,

@@ -456,8 +456,8 @@ cudaError_t layout_build(tsid_template *t, const int32_t *d_rows, const int32_t 
                          const float *d_vals, LayoutScratch &s, int32_t h_flags[FLAG_COUNT]) {
   cudaStream_t st = t->stream;
   const int64_t nnz = t->cfg.nnz;
-  const int32_t m = t->cfg.m, n = t->cfg.n;
-  CK(cudaMemsetAsync(t->flags, 0, sizeof(int32_t) * FLAG_COUNT, st));
+  const int32_t m = t->vm ? t->vm : t->cfg.m, n = t->vn ? t->vn : t->cfg.n;   // a mini-batch template sorts its virtual indices
+  if (!t->n_batches) CK(cudaMemsetAsync(t->flags, 0, sizeof(int32_t) * FLAG_COUNT, st));   // (whose range flag is already set)
   if (nnz > 0) check_coo_kernel<<<grid_for(nnz, 256), 256, 0, st>>>(d_rows, d_cols, nnz, m, n, t->flags);
   CK(cudaGetLastError());
   CK(cudaMemcpyAsync(h_flags, t->flags, sizeof(int32_t) * FLAG_COUNT, cudaMemcpyDeviceToHost, st));

@@ -484,9 +484,15 @@ cudaError_t sparse_grad(tsid_template *t, const float *d_P, const float *d_Q, fl
 }
 
 cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ) {
+  return sparse_update_scaled(t, d_P, d_Q, GP, GQ, t->rowside.scale, t->colside.scale);
+}
+
+// the update with the 2 / s factors taken from the given arrays (one per row of P, one per row of Q)
+cudaError_t sparse_update_scaled(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                                 const float *scale_p, const float *scale_q) {
   const tsid_config_t &c = t->cfg;
-  UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4};
-  UpdSide b{d_Q, GQ, t->colside.scale, t->colside.shadow, (int64_t)c.n * c.k / 4};
+  UpdSide a{d_P, GP, scale_p, t->rowside.shadow, (int64_t)c.m * c.k / 4};
+  UpdSide b{d_Q, GQ, scale_q, t->colside.shadow, (int64_t)c.n * c.k / 4};
   prof_mark(t, EV_UPD0);
   // entry-wise clip: the passes already delivered the sum of clipped per-entry directions (regulariser
   // included), so the update is x += eta * G / s   (scale holds 2 / s)
@@ -611,6 +617,71 @@ cudaError_t sparse_side_sse(tsid_template *t, const Side &sd, const void *stage,
   reduce_slices_kernel<<<RED_BLOCKS, 256, 0, t->stream>>>(warp_part, sd.nseg, sl_a);
   reduce_add_kernel<<<1, 256, 0, t->stream>>>(sl_a, d_out);
   return cudaGetLastError();
+}
+
+// ---- mini-batch template -------------------------------------------------------------------------------
+// rows' = batch * m + row, cols' = batch * n + col; flags[FLAG_RANGE] if a row, column or batch number is out of range
+__global__ void virtual_coo_kernel(const int32_t *__restrict__ rows, const int32_t *__restrict__ cols,
+                                   const int32_t *__restrict__ batch, int64_t nnz, int32_t m, int32_t n, int32_t nb,
+                                   int32_t *__restrict__ vrows, int32_t *__restrict__ vcols, int32_t *flags) {
+  bool bad = false;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nnz; t += (int64_t)gridDim.x * blockDim.x) {
+    const int32_t r = rows[t], c = cols[t], b = batch[t];
+    const bool ok = r >= 0 && r < m && c >= 0 && c < n && b >= 0 && b < nb;
+    bad |= !ok;
+    vrows[t] = ok ? b * m + r : 0;
+    vcols[t] = ok ? b * n + c : 0;
+  }
+  if (bad) flags[FLAG_RANGE] = 1;
+}
+// out[b] = scan[b * stride], b = 0 .. nb
+__global__ void sample_scan_kernel(const uint32_t *__restrict__ scan, int nb, int64_t stride, int32_t *__restrict__ out) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b <= nb; b += gridDim.x * blockDim.x) out[b] = (int32_t)scan[(int64_t)b * stride];
+}
+
+cudaError_t batch_virtual_coo(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols, const int32_t *d_batch) {
+  const tsid_config_t &c = t->cfg;
+  CK(cudaMemsetAsync(t->flags, 0, sizeof(int32_t) * FLAG_COUNT, t->stream));
+  if (c.nnz > 0)
+    virtual_coo_kernel<<<ew_grid(c.nnz), 256, 0, t->stream>>>(d_rows, d_cols, d_batch, c.nnz, c.m, c.n, t->n_batches, t->vrows,
+                                                               t->vcols, t->flags);
+  return cudaGetLastError();
+}
+
+// Right after build_segments of one side: where each batch's segments and split rows begin (the scans of that call are
+// still in the scratch).  The side's rows are the virtual ones, batch b owning [b * rows, (b + 1) * rows).
+cudaError_t batch_ranges(tsid_template *t, const LayoutScratch &s, bool colside) {
+  const int nb = t->n_batches;
+  const int64_t stride = colside ? t->cfg.n : t->cfg.m;
+  int32_t *d_tmp = reinterpret_cast<int32_t *>(s.hist);   // 2 (nb + 1) words of a scratch array nothing else uses now
+  sample_scan_kernel<<<(nb + 256) / 256, 256, 0, t->stream>>>(s.scanA, nb, stride, d_tmp);
+  sample_scan_kernel<<<(nb + 256) / 256, 256, 0, t->stream>>>(s.scanC, nb, stride, d_tmp + nb + 1);
+  CK(cudaGetLastError());
+  CK(cudaMemcpyAsync(colside ? t->bseg_col : t->bseg_row, d_tmp, sizeof(int32_t) * (nb + 1), cudaMemcpyDeviceToHost, t->stream));
+  CK(cudaMemcpyAsync(colside ? t->bsplit_col : t->bsplit_row, d_tmp + nb + 1, sizeof(int32_t) * (nb + 1), cudaMemcpyDeviceToHost,
+                     t->stream));
+  return cudaStreamSynchronize(t->stream);
+}
+
+cudaError_t sparse_batch_step(tsid_template *t, int b, float *d_P, float *d_Q, float *GP, float *GQ) {
+  const tsid_config_t &c = t->cfg;
+  const bool bf = c.precision == TSID_BF16_SHADOW;
+  CK(sparse_convert_shadow(t, d_P, d_Q));
+  const size_t esz = bf ? sizeof(__nv_bfloat16) : sizeof(float);
+  const char *Ps = bf ? reinterpret_cast<const char *>(t->rowside.shadow) : reinterpret_cast<const char *>(d_P);
+  const char *Qs = bf ? reinterpret_cast<const char *>(t->colside.shadow) : reinterpret_cast<const char *>(d_Q);
+  // the layout numbers this batch's rows b * m + i and its columns b * n + j: shift the bases by that many rows so that
+  // the kernels' row arithmetic lands on row i of the real arrays (the shifted pointers are only ever used with those offsets)
+  const ptrdiff_t ro = (ptrdiff_t)b * c.m * c.k, co = (ptrdiff_t)b * c.n * c.k;
+  const void *Pv = Ps - ro * (ptrdiff_t)esz, *Qv = Qs - co * (ptrdiff_t)esz;
+  Side rs = t->rowside, cs = t->colside;
+  rs.segs += t->bseg_row[b]; rs.nseg = t->bseg_row[b + 1] - t->bseg_row[b];
+  rs.splits += t->bsplit_row[b]; rs.nsplit = t->bsplit_row[b + 1] - t->bsplit_row[b];
+  cs.segs += t->bseg_col[b]; cs.nseg = t->bseg_col[b + 1] - t->bseg_col[b];
+  cs.splits += t->bsplit_col[b]; cs.nsplit = t->bsplit_col[b + 1] - t->bsplit_col[b];
+  CK(sparse_side_grad(t, rs, Pv, Qv, GP - ro));
+  CK(sparse_side_grad(t, cs, Qv, Pv, GQ - co));
+  return sparse_update_scaled(t, d_P, d_Q, GP, GQ, t->rowside.scale + (size_t)b * c.m, t->colside.scale + (size_t)b * c.n);
 }
 
 int sparse_launches_per_step(const tsid_template *t) {

@@ -87,6 +87,13 @@ struct tsid_template {
   int32_t *flags;     // device flags: [0] range, [1] unsorted, [2] duplicate, [3] non-finite
   tsid::DenseState *dense;
   tsid::HybridState *hybrid;
+  // Mini-batch template (tsid_template_create_batched): the layout is that of the block-diagonal matrix whose block b
+  // holds batch b, i.e. rows b * m + i and columns b * n + j, so one sort gives (batch, row, col) and (batch, col, row)
+  // order; vm, vn are those virtual sizes (0: an ordinary template).  bseg_* / bsplit_*: first segment / split row of
+  // each batch on either side (host arrays of n_batches + 1 entries).
+  int32_t n_batches, vm, vn;
+  int32_t *bseg_row, *bseg_col, *bsplit_row, *bsplit_col;
+  int32_t *vrows, *vcols;   // device: the virtual COO indices (read by the layout pass only)
   tsid::Prof prof;
   // tsid_fit replays its epochs from an executable graph: fit_steps steps on the factor arrays
   // fit_P / fit_Q, captured on fit_cap (no work ever runs there) and kept until arrays or count change
@@ -168,6 +175,13 @@ cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const ExtendTcMaps *
 cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);
 cudaError_t sparse_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ);
 cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ);
+cudaError_t sparse_update_scaled(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                                 const float *scale_p, const float *scale_q);
+// one batch of a mini-batch template: the passes over the batch's segments (factor and gradient pointers shifted so that
+// the layout's virtual row b * m + i lands on row i), then the update with the batch's own counts
+cudaError_t sparse_batch_step(tsid_template *t, int batch, float *d_P, float *d_Q, float *GP, float *GQ);
+cudaError_t batch_virtual_coo(tsid_template *t, const int32_t *d_rows, const int32_t *d_cols, const int32_t *d_batch);
+cudaError_t batch_ranges(tsid_template *t, const LayoutScratch &s, bool colside);
 cudaError_t sparse_residuals(tsid_template *t, const float *d_P, const float *d_Q, float *d_e);
 cudaError_t sparse_loss(tsid_template *t, const float *d_P, const float *d_Q, double *d_out2);
 int sparse_launches_per_step(const tsid_template *t);

@@ -2,10 +2,12 @@
 
 The paper runs its updates over mini-batches of observed entries (Sec. 5.1: entries are grouped, their
 per-entry updates aggregated per factor row and divided by the number of contributors, Eq. 9).  With this
-library that is the full-batch step applied to one template per batch: Omega is split into `batches` disjoint
-parts, every part gets its own layout, and one epoch is one tsid_grad_step per part, in order, on the same
-P and Q.  The count a row's sum is divided by (TSID_NORM_COUNT) is then the number of ITS entries in the
-batch, which is Eq. 9's n.  The benchmarked path is the full-batch step (batches = 1).
+library that is the full-batch step restricted to a batch: Omega is split into `batches` disjoint parts and one
+epoch is one step per part, in order, on the same P and Q.  The count a row's sum is divided by
+(TSID_NORM_COUNT) is then the number of ITS entries in the batch, which is Eq. 9's n.  Two forms:
+`BatchedTemplate` (ONE library template over all batches: one layout pass, one workspace,
+tsid_grad_step_batch) and the older `MiniBatches` (one template per batch), kept as its cross-check.  The
+benchmarked path is the full-batch step (batches = 1).
 """
 from __future__ import annotations
 
@@ -43,3 +45,28 @@ class MiniBatches:
     def destroy(self):
         for T in self.templates:
             T.tsid_destroy()
+
+
+def batch_ids(nnz: int, batches: int, seed: int, device) -> torch.Tensor:
+    """int32[nnz]: the batch of every entry, the same partition as split_batches gives."""
+    ids = torch.empty(nnz, dtype=torch.int32, device=device)
+    for b, idx in enumerate(split_batches(nnz, batches, seed, device)):
+        ids[idx] = b
+    return ids
+
+
+class BatchedTemplate:
+    """All batches in one library template (tsid_template_create_batched); epoch() steps through them in order."""
+
+    def __init__(self, m, n, k, rows, cols, vals, batches, seed=0, **cfg_kw):
+        self.batches = batches
+        ids = batch_ids(int(rows.numel()), batches, seed, rows.device)
+        cfg = B.make_config(m, n, k, int(rows.numel()), **cfg_kw)
+        self.T = B.Template(cfg, rows, cols, vals, batch=ids, n_batches=batches)
+
+    def epoch(self, P, Q):
+        for b in range(self.batches):
+            self.T.tsid_grad_step_batch(b, P, Q)
+
+    def destroy(self):
+        self.T.tsid_destroy()
