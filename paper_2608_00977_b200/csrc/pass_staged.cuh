@@ -35,6 +35,12 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+// base + j * rowbytes as one multiply-add with a 64-bit addend
+__device__ __forceinline__ const void *row_addr(const unsigned char *base, uint32_t j, uint32_t rowbytes) {
+  uint64_t a;
+  asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(a) : "r"(j), "r"(rowbytes), "l"(reinterpret_cast<uint64_t>(base)));
+  return reinterpret_cast<const void *>(a);
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -128,20 +134,21 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
       const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
       const uint32_t dst0 = sbase + st * STAGE + pp * 16;
       const unsigned char *src0 = reinterpret_cast<const unsigned char *>(gat) + pp * 16;
-      const size_t rowbytes = (size_t)k * sizeof(T);
+      // indices are non-negative: unsigned 32 x 32 + 64 -> 64-bit multiply-add, one instruction per address
       if (k == KP && nv == ROWS) {
 #pragma unroll
         for (int q = 0; q < NCP; ++q) {
           const int r = q * (32 / PIECES) + pr;
-          const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
-          cp_async16(dst0 + r * SLOT, src0 + (size_t)jr * rowbytes);
+          const uint32_t jr = (uint32_t)__shfl_sync(0xffffffffu, j, r & 31);
+          cp_async16(dst0 + r * SLOT, row_addr(src0, jr, (uint32_t)SLOT));
         }
       } else {
+        const uint32_t rowbytes = (uint32_t)k * (uint32_t)sizeof(T);
 #pragma unroll
         for (int q = 0; q < NCP; ++q) {
           const int r = q * (32 / PIECES) + pr;
-          const int32_t jr = __shfl_sync(0xffffffffu, j, r & 31);
-          if (r < nv && pvalid) cp_async16(dst0 + r * SLOT, src0 + (size_t)jr * rowbytes);
+          const uint32_t jr = (uint32_t)__shfl_sync(0xffffffffu, j, r & 31);
+          if (r < nv && pvalid) cp_async16(dst0 + r * SLOT, row_addr(src0, jr, rowbytes));
         }
       }
     }
@@ -184,55 +191,65 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
         const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
         const float myr = vring[u];
         const uint32_t sst = sbase + u * STAGE;
+        // One pair of warp iterations (entries sa and sb = sa + EPW of the chunk) on full-width rows.  Two fp32
+        // FMAs per instruction (sm_100 packed fp32): the dot products run as an even and an odd partial sum,
+        // the accumulation as pairs of coordinates.  FULL: both entries exist.  Otherwise an entry past the
+        // end reads the chunk's last valid row (finite values) and gets e = 0, so it adds nothing.
+        auto pair = [&](auto full, int sa, int sb) {
+          constexpr bool FULL = decltype(full)::value;
+          const bool va = FULL || sa < nv, vb = FULL || sb < nv;
+          if (!FULL) { sa = va ? sa : nv - 1; sb = vb ? sb : nv - 1; }
+          const float ra = __shfl_sync(0xffffffffu, myr, sa);
+          const float rb = __shfl_sync(0xffffffffu, myr, sb);
+          R ya[NV], yb[NV];
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+            SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+          }
+          float fa[EPL], fb[EPL];
+#pragma unroll
+          for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+          float2 da2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fa[0], fa[1]));
+          float2 db2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fb[0], fb[1]));
+#pragma unroll
+          for (int i = 2; i < EPL; i += 2) {
+            const float2 x2 = make_float2(x[i], x[i + 1]);
+            da2 = __ffma2_rn(x2, make_float2(fa[i], fa[i + 1]), da2);
+            db2 = __ffma2_rn(x2, make_float2(fb[i], fb[i + 1]), db2);
+          }
+          float da = da2.x + da2.y, db = db2.x + db2.y;
+#pragma unroll
+          for (int o = GROUP / 2; o > 0; o >>= 1) {
+            da += __shfl_xor_sync(0xffffffffu, da, o);
+            db += __shfl_xor_sync(0xffffffffu, db, o);
+          }
+          const float ea = va ? ra - da : 0.f, eb = vb ? rb - db : 0.f;
+          if (ENTRY) {
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
+          } else {
+            const float2 ea2 = make_float2(ea, ea), eb2 = make_float2(eb, eb);
+#pragma unroll
+            for (int i = 0; i < EPL; i += 2) {
+              float2 a2 = make_float2(acc[i], acc[i + 1]);
+              a2 = __ffma2_rn(ea2, make_float2(fa[i], fa[i + 1]), a2);
+              a2 = __ffma2_rn(eb2, make_float2(fb[i], fb[i + 1]), a2);
+              acc[i] = a2.x;
+              acc[i + 1] = a2.y;
+            }
+          }
+        };
         if (k == KP && nv == ROWS) {
           // full chunk of full-width rows (the common case): no predicates, fully unrolled
 #pragma unroll
-          for (int it = 0; it < ROWS / EPW; it += 2) {
-            const int sa = it * EPW + g, sb = sa + EPW;
-            const float ra = __shfl_sync(0xffffffffu, myr, sa);
-            const float rb = __shfl_sync(0xffffffffu, myr, sb);
-            R ya[NV], yb[NV];
-#pragma unroll
-            for (int q = 0; q < NV; ++q) {
-              SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
-              SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
-            }
-            float fa[EPL], fb[EPL];
-#pragma unroll
-            for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
-            // two fp32 FMAs per instruction (sm_100 packed fp32): the dot products run as an even and an
-            // odd partial sum, the accumulation as pairs of coordinates
-            float2 da2 = make_float2(0.f, 0.f), db2 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int i = 0; i < EPL; i += 2) {
-              const float2 x2 = make_float2(x[i], x[i + 1]);
-              da2 = __ffma2_rn(x2, make_float2(fa[i], fa[i + 1]), da2);
-              db2 = __ffma2_rn(x2, make_float2(fb[i], fb[i + 1]), db2);
-            }
-            float da = da2.x + da2.y, db = db2.x + db2.y;
-#pragma unroll
-            for (int o = GROUP / 2; o > 0; o >>= 1) {
-              da += __shfl_xor_sync(0xffffffffu, da, o);
-              db += __shfl_xor_sync(0xffffffffu, db, o);
-            }
-            const float ea = ra - da, eb = rb - db;
-            if (ENTRY) {
-#pragma unroll
-              for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, true);
-#pragma unroll
-              for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, true);
-            } else {
-              const float2 ea2 = make_float2(ea, ea), eb2 = make_float2(eb, eb);
-#pragma unroll
-              for (int i = 0; i < EPL; i += 2) {
-                float2 a2 = make_float2(acc[i], acc[i + 1]);
-                a2 = __ffma2_rn(ea2, make_float2(fa[i], fa[i + 1]), a2);
-                a2 = __ffma2_rn(eb2, make_float2(fb[i], fb[i + 1]), a2);
-                acc[i] = a2.x;
-                acc[i + 1] = a2.y;
-              }
-            }
-          }
+          for (int it = 0; it < ROWS / EPW; it += 2) pair(std::true_type{}, it * EPW + g, (it + 1) * EPW + g);
+        } else if (k == KP) {
+          // ragged last chunk of a segment
+          const int iters = (nv + EPW - 1) / EPW;
+          for (int it = 0; it < iters; it += 2) pair(std::false_type{}, it * EPW + g, (it + 1) * EPW + g);
         } else {
           const int iters = (nv + EPW - 1) / EPW;
           for (int it = 0; it < iters; it += 2) {
