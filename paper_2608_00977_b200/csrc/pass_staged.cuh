@@ -127,12 +127,12 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
 #pragma unroll
   for (int u = 0; u < NST; ++u) vring[u] = 0.f;
 
-  // Copies of chunk c (lane l < ROWS holds the index of its l-th entry in j) into stage st.
+  // Copies of chunk c (lane l < ROWS holds the index of its l-th entry in j) into the stage at shared address st_addr.
   // Always commits a group, also for chunks past the end, so that wait_group counts stay aligned.
-  auto issue = [&](int c, int st, int32_t j) {
+  auto issue = [&](int c, uint32_t st_addr, int32_t j) {
     if (c < nchunks) {
       const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
-      const uint32_t dst0 = sbase + st * STAGE + pp * 16;
+      const uint32_t dst0 = st_addr + pp * 16;
       const unsigned char *src0 = reinterpret_cast<const unsigned char *>(gat) + pp * 16;
       // indices are non-negative: unsigned 32 x 32 + 64 -> 64-bit multiply-add, one instruction per address
       if (k == KP && nv == ROWS) {
@@ -163,128 +163,156 @@ pass_staged_kernel(const Segment *__restrict__ segs, int nseg, const int32_t *__
     }
   };
 
-  // prologue: chunks 0 .. NST-2 in flight, indices of chunk NST-1 loaded
-  int32_t nj;
-  float nr;
+  // The arithmetic on one landed chunk: stage at shared address sst, values in myr, nv valid entries.
+  auto compute = [&](const uint32_t sst, const float myr, const int nv) {
+    // One pair of warp iterations (entries sa and sb = sa + EPW of the chunk) on full-width rows.  Two fp32
+    // FMAs per instruction (sm_100 packed fp32): the dot products run as an even and an odd partial sum,
+    // the accumulation as pairs of coordinates.  FULL: both entries exist.  Otherwise an entry past the
+    // end reads the chunk's last valid row (finite values) and gets e = 0, so it adds nothing.
+    auto pair = [&](auto full, int sa, int sb) {
+      constexpr bool FULL = decltype(full)::value;
+      const bool va = FULL || sa < nv, vb = FULL || sb < nv;
+      if (!FULL) { sa = va ? sa : nv - 1; sb = vb ? sb : nv - 1; }
+      const float ra = __shfl_sync(0xffffffffu, myr, sa);
+      const float rb = __shfl_sync(0xffffffffu, myr, sb);
+      R ya[NV], yb[NV];
 #pragma unroll
-  for (int u = 0; u < NST - 1; ++u) {
-    int32_t j;
-    load_iv(u, j, vring[u]);
-    issue(u, u, j);
-  }
-  load_iv(NST - 1, nj, nr);
-
-  for (int c0 = 0; c0 < nchunks; c0 += NST) {
+      for (int q = 0; q < NV; ++q) {
+        SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+        SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+      }
+      float fa[EPL], fb[EPL];
 #pragma unroll
-    for (int u = 0; u < NST; ++u) {
-      const int c = c0 + u;
-      if (c < nchunks) {
-        // keep the pipe full: chunk c+NST-1 goes into the stage that chunk c-1 released
-        const int cn = c + NST - 1;
-        const int sn = (u + NST - 1) % NST;
-        vring[sn] = nr;
-        issue(cn, sn, nj);
-        load_iv(cn + 1, nj, nr);
-        cp_async_wait<NST - 1>();  // all but the newest NST-1 groups are done: chunk c has landed
-        __syncwarp();
-
-        const int nv = len - c * ROWS < ROWS ? len - c * ROWS : ROWS;
-        const float myr = vring[u];
-        const uint32_t sst = sbase + u * STAGE;
-        // One pair of warp iterations (entries sa and sb = sa + EPW of the chunk) on full-width rows.  Two fp32
-        // FMAs per instruction (sm_100 packed fp32): the dot products run as an even and an odd partial sum,
-        // the accumulation as pairs of coordinates.  FULL: both entries exist.  Otherwise an entry past the
-        // end reads the chunk's last valid row (finite values) and gets e = 0, so it adds nothing.
-        auto pair = [&](auto full, int sa, int sb) {
-          constexpr bool FULL = decltype(full)::value;
-          const bool va = FULL || sa < nv, vb = FULL || sb < nv;
-          if (!FULL) { sa = va ? sa : nv - 1; sb = vb ? sb : nv - 1; }
-          const float ra = __shfl_sync(0xffffffffu, myr, sa);
-          const float rb = __shfl_sync(0xffffffffu, myr, sb);
-          R ya[NV], yb[NV];
+      for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+      float2 da2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fa[0], fa[1]));
+      float2 db2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fb[0], fb[1]));
 #pragma unroll
-          for (int q = 0; q < NV; ++q) {
-            SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
-            SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
-          }
-          float fa[EPL], fb[EPL];
+      for (int i = 2; i < EPL; i += 2) {
+        const float2 x2 = make_float2(x[i], x[i + 1]);
+        da2 = __ffma2_rn(x2, make_float2(fa[i], fa[i + 1]), da2);
+        db2 = __ffma2_rn(x2, make_float2(fb[i], fb[i + 1]), db2);
+      }
+      float da = da2.x + da2.y, db = db2.x + db2.y;
 #pragma unroll
-          for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
-          float2 da2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fa[0], fa[1]));
-          float2 db2 = __fmul2_rn(make_float2(x[0], x[1]), make_float2(fb[0], fb[1]));
+      for (int o = GROUP / 2; o > 0; o >>= 1) {
+        da += __shfl_xor_sync(0xffffffffu, da, o);
+        db += __shfl_xor_sync(0xffffffffu, db, o);
+      }
+      const float ea = va ? ra - da : 0.f, eb = vb ? rb - db : 0.f;
+      if (ENTRY) {
 #pragma unroll
-          for (int i = 2; i < EPL; i += 2) {
-            const float2 x2 = make_float2(x[i], x[i + 1]);
-            da2 = __ffma2_rn(x2, make_float2(fa[i], fa[i + 1]), da2);
-            db2 = __ffma2_rn(x2, make_float2(fb[i], fb[i + 1]), db2);
-          }
-          float da = da2.x + da2.y, db = db2.x + db2.y;
+        for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
 #pragma unroll
-          for (int o = GROUP / 2; o > 0; o >>= 1) {
-            da += __shfl_xor_sync(0xffffffffu, da, o);
-            db += __shfl_xor_sync(0xffffffffu, db, o);
-          }
-          const float ea = va ? ra - da : 0.f, eb = vb ? rb - db : 0.f;
-          if (ENTRY) {
+        for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
+      } else {
+        const float2 ea2 = make_float2(ea, ea), eb2 = make_float2(eb, eb);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
-#pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
-          } else {
-            const float2 ea2 = make_float2(ea, ea), eb2 = make_float2(eb, eb);
-#pragma unroll
-            for (int i = 0; i < EPL; i += 2) {
-              float2 a2 = make_float2(acc[i], acc[i + 1]);
-              a2 = __ffma2_rn(ea2, make_float2(fa[i], fa[i + 1]), a2);
-              a2 = __ffma2_rn(eb2, make_float2(fb[i], fb[i + 1]), a2);
-              acc[i] = a2.x;
-              acc[i + 1] = a2.y;
-            }
-          }
-        };
-        if (k == KP && nv == ROWS) {
-          // full chunk of full-width rows (the common case): no predicates, fully unrolled
-#pragma unroll
-          for (int it = 0; it < ROWS / EPW; it += 2) pair(std::true_type{}, it * EPW + g, (it + 1) * EPW + g);
-        } else if (k == KP) {
-          // ragged last chunk of a segment
-          const int iters = (nv + EPW - 1) / EPW;
-          for (int it = 0; it < iters; it += 2) pair(std::false_type{}, it * EPW + g, (it + 1) * EPW + g);
-        } else {
-          const int iters = (nv + EPW - 1) / EPW;
-          for (int it = 0; it < iters; it += 2) {
-            const int sa = it * EPW + g, sb = sa + EPW;
-            const float ra = __shfl_sync(0xffffffffu, myr, sa & 31);
-            const float rb = __shfl_sync(0xffffffffu, myr, sb & 31);
-            const bool va = sa < nv, vb = sb < nv;
-            R ya[NV], yb[NV];
-#pragma unroll
-            for (int q = 0; q < NV; ++q) {
-              ya[q].zero();
-              yb[q].zero();
-              if (va && cv[q]) SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
-              if (vb && cv[q]) SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
-            }
-            float fa[EPL], fb[EPL];
-#pragma unroll
-            for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
-            float da = 0.f, db = 0.f;
-#pragma unroll
-            for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
-#pragma unroll
-            for (int o = GROUP / 2; o > 0; o >>= 1) {
-              da += __shfl_xor_sync(0xffffffffu, da, o);
-              db += __shfl_xor_sync(0xffffffffu, db, o);
-            }
-            const float ea = va ? ra - da : 0.f;
-            const float eb = vb ? rb - db : 0.f;
-#pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
-#pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
-          }
+        for (int i = 0; i < EPL; i += 2) {
+          float2 a2 = make_float2(acc[i], acc[i + 1]);
+          a2 = __ffma2_rn(ea2, make_float2(fa[i], fa[i + 1]), a2);
+          a2 = __ffma2_rn(eb2, make_float2(fb[i], fb[i + 1]), a2);
+          acc[i] = a2.x;
+          acc[i + 1] = a2.y;
         }
-        __syncwarp();  // every lane is done reading this stage before it is refilled
+      }
+    };
+    if (k == KP && nv == ROWS) {
+      // full chunk of full-width rows (the common case): no predicates, fully unrolled
+#pragma unroll
+      for (int it = 0; it < ROWS / EPW; it += 2) pair(std::true_type{}, it * EPW + g, (it + 1) * EPW + g);
+    } else if (k == KP) {
+      // ragged last chunk of a segment
+      const int iters = (nv + EPW - 1) / EPW;
+      for (int it = 0; it < iters; it += 2) pair(std::false_type{}, it * EPW + g, (it + 1) * EPW + g);
+    } else {
+      const int iters = (nv + EPW - 1) / EPW;
+      for (int it = 0; it < iters; it += 2) {
+        const int sa = it * EPW + g, sb = sa + EPW;
+        const float ra = __shfl_sync(0xffffffffu, myr, sa & 31);
+        const float rb = __shfl_sync(0xffffffffu, myr, sb & 31);
+        const bool va = sa < nv, vb = sb < nv;
+        R ya[NV], yb[NV];
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+          ya[q].zero();
+          yb[q].zero();
+          if (va && cv[q]) SRaw<BF16, VE>::load(ya[q], sst + sa * SLOT + co[q] * (int)sizeof(T));
+          if (vb && cv[q]) SRaw<BF16, VE>::load(yb[q], sst + sb * SLOT + co[q] * (int)sizeof(T));
+        }
+        float fa[EPL], fb[EPL];
+#pragma unroll
+        for (int q = 0; q < NV; ++q) { ya[q].unpack(fa + q * VE); yb[q].unpack(fb + q * VE); }
+        float da = 0.f, db = 0.f;
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) { da = fmaf(x[i], fa[i], da); db = fmaf(x[i], fb[i], db); }
+#pragma unroll
+        for (int o = GROUP / 2; o > 0; o >>= 1) {
+          da += __shfl_xor_sync(0xffffffffu, da, o);
+          db += __shfl_xor_sync(0xffffffffu, db, o);
+        }
+        const float ea = va ? ra - da : 0.f;
+        const float eb = vb ? rb - db : 0.f;
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(ea, fa[i], x[i], acc[i], lam2, xi, va);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) acc[i] = entry_acc<ENTRY>(eb, fb[i], x[i], acc[i], lam2, xi, vb);
+      }
+    }
+  };
+
+  if (NST == 2) {
+    // two stages: one rolled loop; chunk c is computed while chunk c + 1 lands and the indices and values
+    // of chunk c + 2 are fetched
+    int32_t nj;
+    float nr, rcur;
+    load_iv(0, nj, rcur);
+    issue(0, sbase, nj);
+    load_iv(1, nj, nr);
+    uint32_t scur = sbase, snext = sbase + STAGE;
+    int rem = len;
+    for (int c = 0; c < nchunks; ++c) {
+      const float rnext = nr;
+      issue(c + 1, snext, nj);
+      load_iv(c + 2, nj, nr);
+      cp_async_wait<1>();  // all but the newest group are done: chunk c has landed
+      __syncwarp();
+      compute(scur, rcur, rem < ROWS ? rem : ROWS);
+      __syncwarp();  // every lane is done reading this stage before it is refilled
+      const uint32_t t = scur;
+      scur = snext;
+      snext = t;
+      rcur = rnext;
+      rem -= ROWS;
+    }
+  } else {
+    // prologue: chunks 0 .. NST-2 in flight, indices of chunk NST-1 loaded
+    int32_t nj;
+    float nr;
+  #pragma unroll
+    for (int u = 0; u < NST - 1; ++u) {
+      int32_t j;
+      load_iv(u, j, vring[u]);
+      issue(u, sbase + u * STAGE, j);
+    }
+    load_iv(NST - 1, nj, nr);
+
+    for (int c0 = 0; c0 < nchunks; c0 += NST) {
+  #pragma unroll
+      for (int u = 0; u < NST; ++u) {
+        const int c = c0 + u;
+        if (c < nchunks) {
+          // keep the pipe full: chunk c+NST-1 goes into the stage that chunk c-1 released
+          const int cn = c + NST - 1;
+          const int sn = (u + NST - 1) % NST;
+          vring[sn] = nr;
+          issue(cn, sbase + sn * STAGE, nj);
+          load_iv(cn + 1, nj, nr);
+          cp_async_wait<NST - 1>();  // all but the newest NST-1 groups are done: chunk c has landed
+          __syncwarp();
+
+          compute(sbase + u * STAGE, vring[u], len - c * ROWS < ROWS ? len - c * ROWS : ROWS);
+          __syncwarp();  // every lane is done reading this stage before it is refilled
+        }
       }
     }
   }
