@@ -503,11 +503,9 @@ class StepBench:
                 return sum(a.elapsed_time(b) for a, b in evs)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            if profiled:
-                for _ in range(nsteps):
-                    T.tsid_grad_step(P, Q)
-            else:
-                T.tsid_fit(P, Q, nsteps)      # K steps, replayed from the library's captured graph
+            # K steps of one tsid_fit: replayed from the library's captured graph, or (profiled) the same kernels
+            # launched one by one with the library's events between them
+            T.tsid_fit(P, Q, nsteps)
             b.record(stream)
             self.barrier()
             return a.elapsed_time(b)
@@ -540,7 +538,7 @@ class StepBench:
                 "long_run": long_run, "ms_per_step_with_events": ms_prof,
                 "kernel_ms": {"row_pass": row_ms / nrec, "col_pass": col_ms / nrec, "update": upd_ms / nrec,
                               "tile_passes": tile_ms / nrec},
-                "gpu_launches_per_rep": self.launches * steps if flush else (self.launches - shadow) * steps + shadow,
+                "gpu_launches_per_rep": self.launches * steps if flush else T.tsid_get_fit_launches(steps),
                 "resident_bytes": resident}
 
     def roofline(self, rec, traffic):
@@ -631,7 +629,7 @@ class StepBench:
             fl_alg = 6.0 * 128 * 128 * w.k * tiles   # per step, both tile passes: S, E Y and E^T X of every stored tile
             out["tile_passes"] = {"tiles": tiles, "min_entries_per_tile": min_tile, "entries_in_tiles": nnz - tail,
                                   "ms": km["tile_passes"],
-                                  "what": "rank-ordered shadow copies, tcgen05 tile pass over R tiles and over R^T tiles, two adds",
+                                  "what": "tcgen05 tile pass over R tiles and over R^T tiles (their sums are added by the update kernel, which also keeps the rank-ordered shadow copies current)",
                                   "alg_tflops": fl_alg / (km["tile_passes"] * 1e-3) / 1e12 if km["tile_passes"] else None,
                                   "frac_of_burst_peak": fl_alg / (km["tile_passes"] * 1e-3) / 1e12 / tf_burst if km["tile_passes"] else None}
         return out

@@ -248,6 +248,14 @@ tsid_status_t tsid_residuals(tsid_template_t *t, const float *d_P, const float *
  * tsid_grad_step launches. */
 tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *h_launches_per_step);
 
+/* How many kernels one tsid_fit(t, P, Q, epochs, 0, NULL) enqueues (replayed from a captured graph or
+ * launched one by one, the kernels are the same): the shadow refresh of the call, and per epoch the
+ * passes and the update.  On the hybrid path tsid_fit's epochs launch fewer kernels than tsid_grad_step:
+ * the rank-ordered shadow copies are made once per call and kept current by the update kernel, which also
+ * adds the tile passes' sums to the gather-reduce passes' sums (same order of additions, same bits).
+ * h_launches: host int64. */
+tsid_status_t tsid_get_fit_launches(const tsid_template_t *t, int32_t epochs, int64_t *h_launches);
+
 /* Mini-batch form (Sec. 5.1: the updates run over mini-batches of observed entries, aggregated per factor row and divided
  * by the number of contributors, Eq. 9; a mini-batch step is the full-batch step above restricted to the batch's entries,
  * with Eq. 9's n counted inside the batch).  ONE template holds all batches: d_batch (DEVICE, int32[nnz]) gives the batch of

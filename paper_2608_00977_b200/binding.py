@@ -34,6 +34,7 @@ EXPORTS = ["tsid_workspace_bytes", "tsid_template_create", "tsid_grad_step", "ts
            "tsid_get_pass_times", "tsid_sse_noalloc", "tsid_sample_workspace_bytes", "tsid_sample_template",
            "tsid_extend_workspace_bytes", "tsid_extend", "tsid_grad", "tsid_apply", "tsid_get_counts",
            "tsid_set_norm_counts", "tsid_apply_sliced", "tsid_get_hybrid_info", "tsid_get_step_times",
+           "tsid_get_fit_launches",
            "tsid_debug_stall_tile_pass", "tsid_workspace_bytes_batched", "tsid_template_create_batched",
            "tsid_grad_step_batch"]
 
@@ -88,6 +89,7 @@ def lib():
         L.tsid_get_layout.argtypes = [vp] + [C.POINTER(vp)] * 7
         L.tsid_residuals.argtypes = [vp, vp, vp, vp]
         L.tsid_get_info.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.tsid_get_fit_launches.argtypes = [vp, C.c_int32, C.POINTER(C.c_int64)]
         L.tsid_last_error.argtypes = [vp]
         L.tsid_get_hybrid_info.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
         L.tsid_workspace_bytes_host.argtypes = [C.POINTER(TsidConfig), C.POINTER(C.c_size_t)]
@@ -289,6 +291,13 @@ class Template:
         p, l = C.c_int32(0), C.c_int32(0)
         lib().tsid_get_info(self.h, C.byref(p), C.byref(l))
         return p.value, l.value
+
+    def tsid_get_fit_launches(self, epochs):
+        n = C.c_int64(0)
+        st = lib().tsid_get_fit_launches(self.h, int(epochs), C.byref(n))
+        if st != TSID_OK:
+            self._raise(st)
+        return n.value
 
     def tsid_get_hybrid_info(self):
         """(stored tiles, smallest entry count of a stored tile, entries left to the gather-reduce passes)."""

@@ -109,6 +109,17 @@ cudaError_t grad_any(tsid_template *t, const float *d_P, const float *d_Q, float
   return t->path == TSID_PATH_DENSE_TC ? dense_grad(t, GP, GQ) : sparse_grad(t, d_P, d_Q, GP, GQ);
 }
 
+// One step of tsid_fit on the internal gradient buffers.  The hybrid path leaves the tile passes' sums in their
+// partial blocks and lets the update kernel add them (same order, same bits as hybrid_grad + sparse_update).
+cudaError_t fit_step(tsid_template *t, float *P, float *Q) {
+  if (t->path == TSID_PATH_HYBRID) {
+    cudaError_t e = hybrid_grad_partial(t, t->rowside.G, t->colside.G);
+    return e == cudaSuccess ? hybrid_update(t, P, Q, t->rowside.G, t->colside.G) : e;
+  }
+  cudaError_t e = grad_any(t, P, Q, t->rowside.G, t->colside.G);
+  return e == cudaSuccess ? sparse_update(t, P, Q, t->rowside.G, t->colside.G) : e;
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 tsid_status_t cuda_fail(tsid_template *t, cudaError_t e) {
@@ -143,10 +154,7 @@ cudaError_t fit_graph_get(tsid_template *t, float *P, float *Q, int steps) {
   cudaStream_t user = t->stream;
   t->stream = t->fit_cap;
   cudaError_t el = cudaSuccess;
-  for (int u = 0; u < steps && el == cudaSuccess; ++u) {
-    el = grad_any(t, P, Q, t->rowside.G, t->colside.G);
-    if (el == cudaSuccess) el = sparse_update(t, P, Q, t->rowside.G, t->colside.G);
-  }
+  for (int u = 0; u < steps && el == cudaSuccess; ++u) el = fit_step(t, P, Q);
   t->stream = user;
   cudaGraph_t g = nullptr;
   e = cudaStreamEndCapture(t->fit_cap, &g);
@@ -362,6 +370,7 @@ tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epoch
     if (st != TSID_OK) return st;
   }
   cudaError_t e = sparse_convert_shadow(t, d_P, d_Q);
+  if (e == cudaSuccess && t->path == TSID_PATH_HYBRID) e = hybrid_refresh_ranked(t);
   int ep = 0;
   // a caller that is capturing cfg.stream into a graph of its own gets plain launches
   cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
@@ -381,8 +390,7 @@ tsid_status_t tsid_fit(tsid_template_t *t, float *d_P, float *d_Q, int32_t epoch
   }
   for (; ep < epochs && e == cudaSuccess; ++ep) {
     // the update kernel refreshes the shadows, so they stay current between epochs
-    e = grad_any(t, d_P, d_Q, t->rowside.G, t->colside.G);
-    if (e == cudaSuccess) e = sparse_update(t, d_P, d_Q, t->rowside.G, t->colside.G);
+    e = fit_step(t, d_P, d_Q);
     if (e == cudaSuccess && loss_every > 0 && (ep + 1) % loss_every == 0) {
       st = loss_sync(t, d_P, d_Q, &sse, &sq);
       if (h_sse_history_or_null) h_sse_history_or_null[nh] = sse;
@@ -589,6 +597,15 @@ tsid_status_t tsid_get_info(const tsid_template_t *t, int32_t *h_path, int32_t *
     if (t->path == TSID_PATH_HYBRID) *h_launches_per_step = 1 + hybrid_launches_per_step(t) + 1;   // + shadow refresh, update
     else *h_launches_per_step = t->path == TSID_PATH_DENSE_TC ? dense_launches_per_step(t) : sparse_launches_per_step(t);
   }
+  return TSID_OK;
+}
+
+tsid_status_t tsid_get_fit_launches(const tsid_template_t *t, int32_t epochs, int64_t *h_launches) {
+  if (!t || !h_launches || epochs < 0) return TSID_ERR_INVALID_ARG;
+  const int64_t shadow = t->cfg.precision == TSID_BF16_SHADOW ? 1 : 0;
+  if (t->path == TSID_PATH_HYBRID) *h_launches = shadow + 1 + (int64_t)epochs * (hybrid_launches_per_fit_step(t) + 2);   // one update launch per side
+  else if (t->path == TSID_PATH_DENSE_TC) *h_launches = shadow + (int64_t)epochs * (dense_launches_per_step(t) - shadow);
+  else *h_launches = shadow + (int64_t)epochs * (sparse_launches_per_step(t) - shadow);
   return TSID_OK;
 }
 

@@ -247,7 +247,7 @@ struct HybridState {
   DenseChunk *chunksA = nullptr, *chunksB = nullptr;
   int32_t *rbc = nullptr, *cbc = nullptr;       // first chunk of each row block [IB + 1] / column block [JB + 1]
   int nchA = 0, nchB = 0, capA = 0, capB = 0;
-  float *gpart = nullptr;                       // [max(capA, capB)][128][k] partial gradient blocks
+  float *gpartA = nullptr, *gpartB = nullptr;   // [capA][128][k], [capB][128][k]: sums of the chunks of the two tile passes
   int64_t *tail_row_ptr = nullptr, *tail_col_ptr = nullptr;
   Side tailrow, tailcol;
   alignas(64) unsigned char mapPh[128], mapQh[128], mapRA[128], mapRB[128];
@@ -296,7 +296,8 @@ void hybrid_carve(tsid_template *t, const tsid_config_t &c, Carver &cv) {
   h->ylistA = cv.take<int32_t>(h->max_tiles); h->ylistB = cv.take<int32_t>(h->max_tiles);
   h->chunksA = cv.take<DenseChunk>(h->capA); h->chunksB = cv.take<DenseChunk>(h->capB);
   h->rbc = cv.take<int32_t>(h->IB + 1); h->cbc = cv.take<int32_t>(h->JB + 1);
-  h->gpart = cv.take<float>((size_t)(h->capA > h->capB ? h->capA : h->capB) * HB * k);
+  h->gpartA = cv.take<float>((size_t)h->capA * HB * k);
+  h->gpartB = cv.take<float>((size_t)h->capB * HB * k);
   h->tail_row_ptr = cv.take<int64_t>(m + 1); h->tail_col_ptr = cv.take<int64_t>(n + 1);
   const size_t per = (size_t)c.nnz / kSegLen;
   Side *sides[2] = {&h->tailrow, &h->tailcol};
@@ -471,12 +472,13 @@ void hybrid_info(const tsid_template *t, int64_t *tiles, int32_t *min_entries, i
   *tail = h->nnz_tail;
 }
 
-cudaError_t hybrid_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ) {
-  (void)d_P; (void)d_Q;   // bf16 shadows only
+namespace {
+// tail passes into GP / GQ, tile passes into their partial blocks; with_adds: the blocks are added to GP / GQ too
+cudaError_t hybrid_passes(tsid_template *t, float *GP, float *GQ, bool with_adds) {
   HybridState *h = t->hybrid;
   const tsid_config_t &c = t->cfg;
   cudaStream_t st = t->stream;
-  const int pieces = c.k / 8, k4 = c.k / 4;
+  const int k4 = c.k / 4;
   auto mark = [&](int which) {
     if (t->prof.on && t->prof.nsteps < kProfSteps) cudaEventRecord(t->prof.ev[t->prof.nsteps * EV_PER_STEP + which], st);
   };
@@ -487,17 +489,51 @@ cudaError_t hybrid_grad(tsid_template *t, const float *d_P, const float *d_Q, fl
   CK(sparse_side_grad(t, h->tailcol, t->colside.shadow, t->rowside.shadow, GQ));
   mark(EV_COL1);
   mark(EV_DNS0);
-  gather_rows_kernel<<<grid_for(((int64_t)c.m + c.n) * pieces, 256), 256, 0, st>>>(
-      reinterpret_cast<const uint4 *>(t->rowside.shadow), h->row_of_rank, c.m, reinterpret_cast<uint4 *>(h->Ph),
-      reinterpret_cast<const uint4 *>(t->colside.shadow), h->col_of_rank, c.n, reinterpret_cast<uint4 *>(h->Qh), pieces);
-  CK(dense_tiles_pass(st, c.k, h->Ph, h->mapQh, h->mapRA, h->chunksA, h->nchA, h->ylistA, h->gpart, t->flags));
-  hot_add_kernel<<<dim3(h->IB, 8), 256, 0, st>>>(reinterpret_cast<float4 *>(GP), h->row_of_rank, c.m, k4,
-                                                 reinterpret_cast<const float4 *>(h->gpart), h->rbc);
-  CK(dense_tiles_pass(st, c.k, h->Qh, h->mapPh, h->mapRB, h->chunksB, h->nchB, h->ylistB, h->gpart, t->flags));
-  hot_add_kernel<<<dim3(h->JB, 8), 256, 0, st>>>(reinterpret_cast<float4 *>(GQ), h->col_of_rank, c.n, k4,
-                                                 reinterpret_cast<const float4 *>(h->gpart), h->cbc);
+  CK(dense_tiles_pass(st, c.k, h->Ph, h->mapQh, h->mapRA, h->chunksA, h->nchA, h->ylistA, h->gpartA, t->flags));
+  if (with_adds)
+    hot_add_kernel<<<dim3(h->IB, 8), 256, 0, st>>>(reinterpret_cast<float4 *>(GP), h->row_of_rank, c.m, k4,
+                                                   reinterpret_cast<const float4 *>(h->gpartA), h->rbc);
+  CK(dense_tiles_pass(st, c.k, h->Qh, h->mapPh, h->mapRB, h->chunksB, h->nchB, h->ylistB, h->gpartB, t->flags));
+  if (with_adds)
+    hot_add_kernel<<<dim3(h->JB, 8), 256, 0, st>>>(reinterpret_cast<float4 *>(GQ), h->col_of_rank, c.n, k4,
+                                                   reinterpret_cast<const float4 *>(h->gpartB), h->cbc);
   mark(EV_DNS1);
   return cudaGetLastError();
+}
+}  // namespace
+
+// rank-ordered copies of the current bf16 shadows
+cudaError_t hybrid_refresh_ranked(tsid_template *t) {
+  HybridState *h = t->hybrid;
+  const tsid_config_t &c = t->cfg;
+  const int pieces = c.k / 8;
+  gather_rows_kernel<<<grid_for(((int64_t)c.m + c.n) * pieces, 256), 256, 0, t->stream>>>(
+      reinterpret_cast<const uint4 *>(t->rowside.shadow), h->row_of_rank, c.m, reinterpret_cast<uint4 *>(h->Ph),
+      reinterpret_cast<const uint4 *>(t->colside.shadow), h->col_of_rank, c.n, reinterpret_cast<uint4 *>(h->Qh), pieces);
+  return cudaGetLastError();
+}
+
+// complete gradient sums in GP / GQ (what tsid_grad_step and tsid_grad hand out)
+cudaError_t hybrid_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ) {
+  (void)d_P; (void)d_Q;   // bf16 shadows only
+  CK(hybrid_refresh_ranked(t));
+  return hybrid_passes(t, GP, GQ, true);
+}
+
+cudaError_t hybrid_grad_partial(tsid_template *t, float *GP, float *GQ) { return hybrid_passes(t, GP, GQ, false); }
+
+cudaError_t hybrid_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ) {
+  HybridState *h = t->hybrid;
+  UpdHot hp, hq;
+  hp.rank_of = h->rank_of_row; hp.first_chunk = h->rbc; hp.part = h->gpartA; hp.ranked = h->Ph;
+  hq.rank_of = h->rank_of_col; hq.first_chunk = h->cbc; hq.part = h->gpartB; hq.ranked = h->Qh;
+  return sparse_update_hot(t, d_P, d_Q, GP, GQ, hp, hq);
+}
+
+// tail passes (+ fix-ups) + two tile-list passes; the update kernel is counted by the caller
+int hybrid_launches_per_fit_step(const tsid_template *t) {
+  const HybridState *h = t->hybrid;
+  return 2 + (h->tailrow.nsplit > 0) + (h->tailcol.nsplit > 0) + 2;
 }
 
 }  // namespace tsid

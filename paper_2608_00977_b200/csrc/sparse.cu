@@ -212,6 +212,7 @@ struct UpdSide {
   const float *scale;
   __nv_bfloat16 *shadow;
   int64_t n4;  // rows * k / 4
+  UpdHot hot;  // hybrid path: sums of the tile passes still to be added, rank-ordered shadow copy
 };
 
 __device__ __forceinline__ float clip_dir(float d, float xi, int clip) {
@@ -221,18 +222,35 @@ __device__ __forceinline__ float clip_dir(float d, float xi, int clip) {
 }
 
 // D = G * (2/s) - 2 lambda X; clip; X += eta D; refresh the bf16 shadow; flag non-finite values.
-__global__ void __launch_bounds__(256)
+// HOT: the side carries sums of the hybrid path's tile passes (UpdHot); launched per side (side b unused), which
+// keeps it at 48 registers.
+template <bool HOT>
+__global__ void __launch_bounds__(256, HOT ? 5 : 8)
 update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int clip, float gmul, int32_t *flags) {
-  const int64_t total = a.n4 + b.n4;
+  const int64_t total = HOT ? a.n4 : a.n4 + b.n4;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   bool bad = false;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-    const bool first = i < a.n4;
+    const bool first = HOT || i < a.n4;
     const UpdSide &sd = first ? a : b;
     const int64_t j = first ? i : i - a.n4;
     const float sc = __ldg(sd.scale + j / k4) * gmul;
     float4 x = reinterpret_cast<float4 *>(sd.X)[j];
-    const float4 gv = __ldcs(reinterpret_cast<const float4 *>(sd.G) + j);
+    float4 gv = __ldcs(reinterpret_cast<const float4 *>(sd.G) + j);
+    int r = 0;
+    if (HOT && sd.hot.rank_of) {
+      // + the sums of the row block's chunks, added among themselves first, in chunk order
+      r = __ldg(sd.hot.rank_of + j / k4);
+      const int l = (int)(j % k4), c0 = __ldg(sd.hot.first_chunk + (r >> 7)), c1 = __ldg(sd.hot.first_chunk + (r >> 7) + 1);
+      if (c1 > c0) {
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = c0; c < c1; ++c) {
+          const float4 p = __ldcs(reinterpret_cast<const float4 *>(sd.hot.part) + ((size_t)c * 128 + (r & 127)) * k4 + l);
+          sum.x += p.x; sum.y += p.y; sum.z += p.z; sum.w += p.w;
+        }
+        gv.x += sum.x; gv.y += sum.y; gv.z += sum.z; gv.w += sum.w;
+      }
+    }
     float xs[4] = {x.x, x.y, x.z, x.w};
     const float gs[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
@@ -251,6 +269,7 @@ update_kernel(UpdSide a, UpdSide b, int k4, float eta, float lam2, float xi, int
       pk.x = *reinterpret_cast<uint32_t *>(&lo);
       pk.y = *reinterpret_cast<uint32_t *>(&hi);
       reinterpret_cast<uint2 *>(sd.shadow)[j] = pk;
+      if (HOT && sd.hot.ranked) reinterpret_cast<uint2 *>(sd.hot.ranked)[(size_t)r * k4 + j % k4] = pk;
     }
   }
   if (bad) flags[FLAG_NONFINITE] = 1;
@@ -487,19 +506,41 @@ cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float 
   return sparse_update_scaled(t, d_P, d_Q, GP, GQ, t->rowside.scale, t->colside.scale);
 }
 
+cudaError_t update_launch(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                          const float *scale_p, const float *scale_q, const UpdHot &hot_p, const UpdHot &hot_q);
+
 // the update with the 2 / s factors taken from the given arrays (one per row of P, one per row of Q)
 cudaError_t sparse_update_scaled(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
                                  const float *scale_p, const float *scale_q) {
+  return update_launch(t, d_P, d_Q, GP, GQ, scale_p, scale_q, UpdHot(), UpdHot());
+}
+
+// the update that also adds the hybrid path's tile sums (see UpdHot)
+cudaError_t sparse_update_hot(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                              const UpdHot &hot_p, const UpdHot &hot_q) {
+  return update_launch(t, d_P, d_Q, GP, GQ, t->rowside.scale, t->colside.scale, hot_p, hot_q);
+}
+
+cudaError_t update_launch(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                          const float *scale_p, const float *scale_q, const UpdHot &hot_p, const UpdHot &hot_q) {
   const tsid_config_t &c = t->cfg;
-  UpdSide a{d_P, GP, scale_p, t->rowside.shadow, (int64_t)c.m * c.k / 4};
-  UpdSide b{d_Q, GQ, scale_q, t->colside.shadow, (int64_t)c.n * c.k / 4};
+  UpdSide a{d_P, GP, scale_p, t->rowside.shadow, (int64_t)c.m * c.k / 4, hot_p};
+  UpdSide b{d_Q, GQ, scale_q, t->colside.shadow, (int64_t)c.n * c.k / 4, hot_q};
   prof_mark(t, EV_UPD0);
   // entry-wise clip: the passes already delivered the sum of clipped per-entry directions (regulariser
   // included), so the update is x += eta * G / s   (scale holds 2 / s)
   const bool entry = c.clip == TSID_CLIP_ASYM_ENTRY;
-  update_kernel<<<ew_grid(a.n4 + b.n4), 256, 0, t->stream>>>(a, b, c.k / 4, c.eta, entry ? 0.f : 2.0f * c.lambda, c.xi,
-                                                             entry ? (int)TSID_CLIP_NONE : c.clip, entry ? 0.5f : 1.0f,
-                                                             t->flags);
+  if (hot_p.rank_of || hot_q.rank_of) {
+    if (a.n4 > 0)
+      update_kernel<true><<<ew_grid(a.n4), 256, 0, t->stream>>>(a, a, c.k / 4, c.eta, entry ? 0.f : 2.0f * c.lambda, c.xi,
+                                                                entry ? (int)TSID_CLIP_NONE : c.clip, entry ? 0.5f : 1.0f, t->flags);
+    if (b.n4 > 0)
+      update_kernel<true><<<ew_grid(b.n4), 256, 0, t->stream>>>(b, b, c.k / 4, c.eta, entry ? 0.f : 2.0f * c.lambda, c.xi,
+                                                                entry ? (int)TSID_CLIP_NONE : c.clip, entry ? 0.5f : 1.0f, t->flags);
+  } else
+    update_kernel<false><<<ew_grid(a.n4 + b.n4), 256, 0, t->stream>>>(a, b, c.k / 4, c.eta, entry ? 0.f : 2.0f * c.lambda, c.xi,
+                                                                      entry ? (int)TSID_CLIP_NONE : c.clip, entry ? 0.5f : 1.0f,
+                                                                      t->flags);
   prof_mark(t, EV_UPD1);
   if (t->prof.on && t->prof.nsteps < kProfSteps) t->prof.nsteps++;
   return cudaGetLastError();
@@ -560,10 +601,10 @@ cudaError_t sparse_apply_sliced(tsid_template *t, float *d_P, const float *GP, f
   const bool entry = c.clip == TSID_CLIP_ASYM_ENTRY;
   const float lam2 = entry ? 0.f : 2.0f * c.lambda, gmul = entry ? 0.5f : 1.0f;
   const int clip = entry ? (int)TSID_CLIP_NONE : (int)c.clip;
-  UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4};
-  UpdSide none{nullptr, nullptr, nullptr, nullptr, 0};
+  UpdSide a{d_P, GP, t->rowside.scale, t->rowside.shadow, (int64_t)c.m * c.k / 4, UpdHot()};
+  UpdSide none{nullptr, nullptr, nullptr, nullptr, 0, UpdHot()};
   prof_mark(t, EV_UPD0);
-  if (a.n4 > 0) update_kernel<<<ew_grid(a.n4), 256, 0, t->stream>>>(a, none, c.k / 4, c.eta, lam2, c.xi, clip, gmul, t->flags);
+  if (a.n4 > 0) update_kernel<false><<<ew_grid(a.n4), 256, 0, t->stream>>>(a, none, c.k / 4, c.eta, lam2, c.xi, clip, gmul, t->flags);
   PeerPtrs pp;
   for (int r = 0; r < kMaxPeers; ++r) { pp.gq[r] = nullptr; pp.q[r] = nullptr; }
   for (int r = 0; r < world; ++r) { pp.gq[r] = h_GQ[r]; pp.q[r] = h_Q[r]; }

@@ -175,6 +175,18 @@ cudaError_t extend_tc_adam(cudaStream_t st, const float *U, const ExtendTcMaps *
 cudaError_t sparse_convert_shadow(tsid_template *t, const float *d_P, const float *d_Q);
 cudaError_t sparse_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ);
 cudaError_t sparse_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ);
+// What the update kernel adds to one side when the tile passes of the hybrid path left their sums in partial
+// blocks: row i has popularity rank r = rank_of[i]; the chunks [first_chunk[r / 128], first_chunk[r / 128 + 1]) of
+// its block hold row r % 128 of their sums; `ranked` (or null) is the rank-ordered copy of the bf16 shadow,
+// refreshed in the same kernel.
+struct UpdHot {
+  const int32_t *rank_of = nullptr;
+  const int32_t *first_chunk = nullptr;
+  const float *part = nullptr;
+  __nv_bfloat16 *ranked = nullptr;
+};
+cudaError_t sparse_update_hot(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
+                              const UpdHot &hot_p, const UpdHot &hot_q);
 cudaError_t sparse_update_scaled(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ,
                                  const float *scale_p, const float *scale_q);
 // one batch of a mini-batch template: the passes over the batch's segments (factor and gradient pointers shifted so that
@@ -219,6 +231,13 @@ void hybrid_carve(tsid_template *t, const tsid_config_t &c, Carver &cv);
 // builds the tiles and the tail layout; *h_status: 0 ok, 1 no tile worth it (or duplicates / fp16 range): run sparse
 cudaError_t hybrid_build(tsid_template *t, LayoutScratch &s, int32_t *h_status);
 cudaError_t hybrid_grad(tsid_template *t, const float *d_P, const float *d_Q, float *GP, float *GQ);
+// The step as tsid_fit runs it: hybrid_refresh_ranked once after the shadows were refreshed, then per step
+// hybrid_grad_partial (tail sums in GP / GQ, tile sums left in their partial blocks) and hybrid_update (which adds
+// the two in the order hybrid_grad adds them and keeps the rank-ordered shadow copies current).
+cudaError_t hybrid_refresh_ranked(tsid_template *t);
+cudaError_t hybrid_grad_partial(tsid_template *t, float *GP, float *GQ);
+cudaError_t hybrid_update(tsid_template *t, float *d_P, float *d_Q, const float *GP, const float *GQ);
+int hybrid_launches_per_fit_step(const tsid_template *t);
 int hybrid_launches_per_step(const tsid_template *t);
 void hybrid_info(const tsid_template *t, int64_t *tiles, int32_t *min_entries, int64_t *tail);
 

@@ -118,7 +118,14 @@ def test_hybrid_trajectory_rmse_determinism_and_graph_replay():
     for _ in range(w.epochs):
         T.tsid_grad_step(P3, Q3)
     assert torch.equal(P3, P) and torch.equal(Q3, Q)
+    # tsid_fit's epochs leave the tile sums to the update kernel and keep the rank-ordered shadow copies current
+    # there (one launch per side): per epoch three kernels fewer than tsid_grad_step, the same bits (above)
+    per_step = T.tsid_get_info()[1]
+    assert T.tsid_get_fit_launches(w.epochs) == 2 + w.epochs * (per_step - 3)
     T.tsid_destroy()
+    Ts = B.template_from_workload(tpl, path=B.TSID_PATH_SPARSE)
+    assert Ts.tsid_get_fit_launches(5) == 1 + 5 * (Ts.tsid_get_info()[1] - 1)
+    Ts.tsid_destroy()
     T2 = B.template_from_workload(tpl, path=B.TSID_PATH_HYBRID)       # a second handle: same bits
     P4, Q4 = tpl.P0.clone(), tpl.Q0.clone()
     T2.tsid_fit(P4, Q4, w.epochs)
