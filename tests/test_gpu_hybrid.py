@@ -99,8 +99,9 @@ def test_hybrid_step_against_oracle_and_sparse_path(k):
     assert relerr(d[0], s[0]) <= 1e-2 and relerr(d[1], s[1]) <= 1e-2
 
 
-def test_hybrid_trajectory_rmse_determinism_and_graph_replay():
-    w = _zipf(128, seed=91)
+@pytest.mark.parametrize("k", [128, 64])
+def test_hybrid_trajectory_rmse_determinism_and_graph_replay(k):
+    w = _zipf(k, seed=91)
     tpl = W.make_template(w, DEV)
     r, c, v = np_coo(tpl)
     P0, Q0 = tpl.P0.cpu().numpy(), tpl.Q0.cpu().numpy()
