@@ -80,6 +80,13 @@ def _sampled_check(w, path, tol_g, n_random=4096, n_hot=16, emulate=True, tol_tr
         sse_ref, _ = oracle.loss(len(sample), Y.shape[0], w.k, sub_r, sub_c, sub_v, Xs, Y, 0.0, bf16_emulate=emulate)
         assert len(sub_r) == pos.numel() and abs(sse_gpu - sse_ref) <= 1e-5 * sse_ref, (side, sse_gpu, sse_ref)
         del seg, pos
+    # one epoch of tsid_fit from the same factors ends on the same bits as the tsid_grad_step above (on the hybrid
+    # path the fit leaves the tile passes' sums to the update kernel)
+    del GP, GQ, e_csr
+    P2, Q2 = tpl.P0.clone(), tpl.Q0.clone()
+    T.tsid_fit(P2, Q2, 1)
+    T.tsid_check()
+    assert torch.equal(P2, P) and torch.equal(Q2, Q)
     T.tsid_destroy()
     return got_path, worst
 
